@@ -1,0 +1,132 @@
+"""ctypes access to the C++ CPU oracle (oracle/falcon_oracle.cpp).
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, by the smoke check and by the
+benchmark's CPU-baseline leg.  The product package never imports this.
+Arguments are numpy arrays; bf16 tensors travel as uint16 bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes as C
+
+import numpy as np
+
+from .build_oracle import build as _build
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(_build())
+        _lib.oracle_max_threads.restype = C.c_int
+    return _lib
+
+
+def _p(a, ctype):
+    return None if a is None else a.ctypes.data_as(C.POINTER(ctype))
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def max_threads() -> int:
+    return int(lib().oracle_max_threads())
+
+
+def tree_validate(parent) -> int:
+    parent = _i32(parent)
+    return int(lib().oracle_tree_validate(_p(parent, C.c_int32), C.c_int32(len(parent))))
+
+
+def ancestors(parent, i: int):
+    parent = _i32(parent)
+    out = np.empty(len(parent) + 1, dtype=np.int32)
+    n = lib().oracle_ancestors(_p(parent, C.c_int32), C.c_int32(len(parent)), C.c_int32(i), _p(out, C.c_int32))
+    if n < 0:
+        raise ValueError("malformed tree")
+    return out[:n].copy()
+
+
+def tree_attn(node_off, parent, prefix_len, Hq, Hkv, D, sm_scale, q, k_cache, v_cache, strides,
+              k_tree=None, v_tree=None, tree_mask=None, n_threads=0):
+    """fp32 [N, Hq, D] attention output.  strides = (b, h, s) in elements."""
+    node_off, parent, prefix_len = _i32(node_off), _i32(parent), _i32(prefix_len)
+    N = int(node_off[-1])
+    out = np.empty((N, Hq, D), dtype=np.float32)
+    assert q.dtype == np.uint16 and k_cache.dtype == np.uint16 and v_cache.dtype == np.uint16
+    if tree_mask is not None:
+        tree_mask = np.ascontiguousarray(tree_mask, dtype=np.uint64)
+        assert tree_mask.shape == (N, 2)
+    rc = lib().oracle_tree_attn(
+        C.c_int32(len(prefix_len)), _p(node_off, C.c_int32), _p(parent, C.c_int32), _p(prefix_len, C.c_int32),
+        C.c_int32(Hq), C.c_int32(Hkv), C.c_int32(D), C.c_float(sm_scale), _p(q, C.c_uint16),
+        _p(k_cache, C.c_uint16), _p(v_cache, C.c_uint16), C.c_int64(strides[0]), C.c_int64(strides[1]),
+        C.c_int64(strides[2]), _p(k_tree, C.c_uint16), _p(v_tree, C.c_uint16), _p(tree_mask, C.c_uint64),
+        _p(out, C.c_float), C.c_int(n_threads))
+    if rc:
+        raise ValueError("oracle_tree_attn failed: %d" % rc)
+    return out
+
+
+def causal_attn(L, T, Hq, Hkv, D, sm_scale, q, k, v):
+    out = np.empty((T, Hq, D), dtype=np.float32)
+    q, k, v = (np.ascontiguousarray(a, dtype=np.uint16) for a in (q, k, v))
+    assert k.shape == (Hkv, L + T, D) and v.shape == k.shape and q.shape == (T, Hq, D)
+    rc = lib().oracle_causal_attn(C.c_int32(L), C.c_int32(T), C.c_int32(Hq), C.c_int32(Hkv), C.c_int32(D),
+                                  C.c_float(sm_scale), _p(q, C.c_uint16), _p(k, C.c_uint16), _p(v, C.c_uint16),
+                                  _p(out, C.c_float))
+    if rc:
+        raise ValueError("oracle_causal_attn failed: %d" % rc)
+    return out
+
+
+def argmax(logits, vocab=None, n_threads=0):
+    """logits: C-contiguous fp32 [N, stride]; the first `vocab` columns of each row are scanned."""
+    assert logits.dtype == np.float32 and logits.ndim == 2 and logits.flags.c_contiguous
+    N, stride = logits.shape
+    V = stride if vocab is None else vocab
+    g = np.empty(N, dtype=np.int32)
+    rc = lib().oracle_argmax(_p(logits, C.c_float), C.c_int32(N), C.c_int32(V), C.c_int64(stride),
+                             _p(g, C.c_int32), C.c_int(n_threads))
+    if rc:
+        raise ValueError("oracle_argmax failed: %d" % rc)
+    return g
+
+
+def _accept(fn, node_off, parent, token, g, path_stride):
+    node_off, parent, token, g = _i32(node_off), _i32(parent), _i32(token), _i32(g)
+    B = len(node_off) - 1
+    path = np.empty((B, path_stride), dtype=np.int32)
+    n_path = np.empty(B, dtype=np.int32)
+    nxt = np.empty(B, dtype=np.int32)
+    rc = fn(C.c_int32(B), _p(node_off, C.c_int32), _p(parent, C.c_int32), _p(token, C.c_int32), _p(g, C.c_int32),
+            _p(path, C.c_int32), C.c_int32(path_stride), _p(n_path, C.c_int32), _p(nxt, C.c_int32))
+    if rc:
+        raise ValueError("oracle accept failed: %d" % rc)
+    return path, n_path, nxt
+
+
+def tree_accept(node_off, parent, token, g, path_stride=128):
+    return _accept(lib().oracle_tree_accept, node_off, parent, token, g, path_stride)
+
+
+def bruteforce_accept(node_off, parent, token, g, path_stride=128):
+    return _accept(lib().oracle_bruteforce_accept, node_off, parent, token, g, path_stride)
+
+
+def kv_compact(node_off, prefix_len, Hkv, D, cache, strides, s_cap, path, n_path, tree_rows=None):
+    """Compacts `cache` (uint16 numpy array, modified in place); returns new_len."""
+    node_off, prefix_len, n_path = _i32(node_off), _i32(prefix_len), _i32(n_path)
+    path = np.ascontiguousarray(path, dtype=np.int32)
+    assert cache.dtype == np.uint16 and cache.flags.c_contiguous
+    new_len = np.empty(len(prefix_len), dtype=np.int32)
+    rc = lib().oracle_kv_compact(
+        C.c_int32(len(prefix_len)), _p(node_off, C.c_int32), _p(prefix_len, C.c_int32), C.c_int32(Hkv),
+        C.c_int32(D), _p(cache, C.c_uint16), C.c_int64(strides[0]), C.c_int64(strides[1]), C.c_int64(strides[2]),
+        C.c_int32(s_cap), _p(tree_rows, C.c_uint16), _p(path, C.c_int32), C.c_int32(path.shape[1]),
+        _p(n_path, C.c_int32), _p(new_len, C.c_int32))
+    if rc:
+        raise ValueError("oracle_kv_compact failed: %d" % rc)
+    return new_len
