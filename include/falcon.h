@@ -1,0 +1,192 @@
+/*
+ * falcon.h - C ABI of the tree-verification step of Falcon speculative decoding
+ * (arXiv 2412.12639) for NVIDIA B200 (sm_100a).
+ *
+ * One verification step of the target model over the decoding tree is
+ *     n_layers x falcon_tree_attn  ->  falcon_tree_accept  ->  falcon_kv_compact
+ * (Section 3.4: the drafts form a token tree that the target model verifies in
+ * one parallel pass, then "the accepted tokens and their corresponding
+ * features" are recorded for the next drafting phase; Section 4.1: greedy
+ * decoding, temperature 0).
+ *
+ * General rules
+ *   - Every pointer inside an *_args struct is a DEVICE pointer unless its name
+ *     ends in _host.  The structs themselves are host memory and are read
+ *     before the call returns.  The caller owns every buffer; the library owns
+ *     only the falcon_ctx (scratch memory, cached TMA descriptors).
+ *   - `stream` is a cudaStream_t passed as void*.  All work is enqueued on it;
+ *     no call synchronises.  A context must not be used from two streams at
+ *     the same time (its scratch memory is shared by its calls).
+ *   - Return value: FALCON_OK or an error code; on error nothing was launched.
+ *   - Faults only the device can see (a malformed parent array, a tree that
+ *     does not fit the cache) never trap: the kernel clamps the access, skips
+ *     the sequence's result where it must, and ORs FALCON_DEV_* bits into the
+ *     optional per-sequence device word tree.status[b].
+ *   - The first call of each kind on a context may allocate scratch memory
+ *     (cudaMalloc); make that call before capturing the stream into a graph.
+ *   - There is no CPU fallback and no alternative backend.
+ *
+ * Tree convention (Section 3.4, Appendix A): a sequence's tree has T <=
+ * FALCON_T_MAX single-token nodes with local indices 0..T-1, node 0 is the
+ * root (the token the target model has already emitted; a k-token root is a
+ * chain of k nodes), parent[0] = -1 and 0 <= parent[i] < i.  Batches are
+ * packed: sequence b owns nodes node_off[b] .. node_off[b+1]-1.
+ */
+#ifndef FALCON_H_
+#define FALCON_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FALCON_T_MAX 128
+
+enum {
+  FALCON_OK = 0,
+  FALCON_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, bad stride          */
+  FALCON_ERR_UNSUPPORTED = 2, /* head_dim not 64/128, tree > FALCON_T_MAX, Hq % Hkv   */
+  FALCON_ERR_CUDA = 3,        /* a CUDA runtime/driver call failed                    */
+  FALCON_ERR_BAD_TREE = 4,    /* host-side tree validation failed                     */
+  FALCON_ERR_CAPACITY = 5,    /* sizes exceed a stated maximum                        */
+  FALCON_ERR_TIMEOUT = 6      /* a bounded device wait gave up (reported via status)  */
+};
+
+/* bits of the optional device status word tree.status[b] */
+enum {
+  FALCON_DEV_BAD_TREE = 1, /* parent[0] != -1 or parent[i] outside [0, i)            */
+  FALCON_DEV_CAPACITY = 2, /* prefix_len + tree size exceeds s_cap                   */
+  FALCON_DEV_BAD_PATH = 4, /* path / n_path entry outside the tree (compaction)      */
+  FALCON_DEV_TIMEOUT = 8   /* a bounded wait on an on-chip barrier ran out           */
+};
+
+typedef struct falcon_ctx falcon_ctx;
+
+/* Creates a context on CUDA device `device` (made current for the call). */
+int falcon_create(falcon_ctx** out, int device);
+/* Frees the context's scratch memory.  The caller makes sure no work is in flight. */
+int falcon_destroy(falcon_ctx* ctx);
+/* Static, human-readable name of a return code. */
+const char* falcon_status_string(int status);
+/* Text of the last CUDA error seen by this context ("" if none). */
+const char* falcon_last_error(const falcon_ctx* ctx);
+/* Host check of one tree: FALCON_OK iff T in [1, FALCON_T_MAX], parent[0] == -1
+ * and 0 <= parent[i] < i.  `parent` is a HOST pointer. */
+int falcon_tree_validate_host(const int32_t* parent, int32_t T);
+
+/* Packed description of the batch of trees shared by the three calls. */
+typedef struct {
+  int32_t batch;                  /* B >= 1                                             */
+  int32_t total_nodes;            /* N = sum of tree sizes (host knows it)              */
+  int32_t max_tree;               /* max tree size, <= FALCON_T_MAX                     */
+  int32_t max_prefix_len;         /* host upper bound on prefix_len[b] (grid sizing)    */
+  const int32_t* node_off;        /* [B+1] node_off[0] = 0                              */
+  const int32_t* parent;          /* [N] local parent index, -1 at each local node 0    */
+  const int32_t* token;           /* [N] drafted token ids (used by accept only)        */
+  const int32_t* prefix_len;      /* [B] rows of the cache that hold the prefix         */
+  const int32_t* prefix_len_host; /* optional HOST copy of prefix_len (scheduling hint) */
+  int32_t* status;                /* optional [B] device status words (FALCON_DEV_*)    */
+} falcon_tree_desc;
+
+/* ---------------------------------------------------------------------------
+ * falcon_tree_attn - tree-masked attention of ONE layer (Section 3.4: the target
+ * model scores all tree tokens in one pass with tree attention, each token
+ * seeing the prefix and its predecessors in the tree; Section 4.5).
+ *
+ * For node i of sequence b and query head h (KV head h / (Hq/Hkv)):
+ *   keys     {0..L_b-1}  U  {L_b + t : t ancestor-or-self of i}
+ *   out[i,h] = softmax_j(sm_scale * q[i,h].K[j]) . V[j]    (fp32 accumulate)
+ * tree_mask, when given, replaces "ancestor-or-self" by the set bits of a
+ * caller-supplied row (the drafter's relaxed causal mask of Section 3.4).
+ *
+ * q, out      bf16 [N, Hq, D] contiguous, 16-byte aligned.
+ * k/v_cache   bf16, D contiguous, element strides kv_stride_{b,h,s}; row L_b+t
+ *             of sequence b holds tree node t's K/V unless k_tree/v_tree given.
+ *             Base 16-byte aligned, strides multiples of 8 elements.
+ * k/v_tree    optional bf16 [N, Hkv, D]: tree K/V kept outside the cache.
+ * kernel      FALCON_ATTN_AUTO picks; the others force one kernel (tests).
+ * n_splits    0 = automatic; else the number of KV splits per head (1..8 for
+ *             the tensor-core kernel, 1..64 for the SIMT kernel).
+ * ------------------------------------------------------------------------- */
+enum { FALCON_ATTN_AUTO = 0, FALCON_ATTN_SIMT = 1, FALCON_ATTN_TC = 2 };
+
+typedef struct {
+  falcon_tree_desc tree;
+  int32_t n_q_heads, n_kv_heads, head_dim; /* Hq % Hkv == 0; D in {64, 128}            */
+  float sm_scale;                          /* usually 1/sqrt(D)                         */
+  const void* q;
+  void* out;
+  const void* k_cache;
+  const void* v_cache;
+  int64_t kv_stride_b, kv_stride_h, kv_stride_s;
+  int32_t s_cap;                           /* rows per (sequence, head) in the cache    */
+  const void* k_tree;
+  const void* v_tree;
+  const uint64_t* tree_mask;               /* optional [N][2]: bit t of row i = node i sees tree key t */
+  int32_t kernel;
+  int32_t n_splits;
+} falcon_attn_args;
+
+int falcon_tree_attn(falcon_ctx* ctx, const falcon_attn_args* args, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * falcon_tree_accept - greedy acceptance (Section 4.1 temperature 0; Section 3.4
+ * verification as in SpecInfer; the accepted length is tau of Section 4.2).
+ *
+ *   g[i]      = lowest index of the maximum of logits[i, 0..V-1]  (NaN never wins;
+ *               a row with nothing above -inf gives 0)
+ *   alive(c)  = every non-root node a on the root..c chain has token[a] == g[parent[a]]
+ *   result    = alive node of greatest depth, lowest index among equals
+ *   path[b]   = its root-to-node chain (local indices, path[b][0] == 0, rest -1)
+ *   n_path[b] = nodes on the path (accepted drafted tokens = n_path - 1)
+ *   next_token[b] = g[last node of the path]
+ * ------------------------------------------------------------------------- */
+typedef struct {
+  falcon_tree_desc tree;
+  int32_t vocab;
+  int64_t logits_stride;  /* elements between rows, >= vocab                          */
+  const float* logits;    /* fp32 [N, logits_stride]                                  */
+  int32_t* argmax_out;    /* [N] g, always written                                    */
+  int32_t* path;          /* [B, path_stride]                                         */
+  int32_t path_stride;    /* >= max_tree                                              */
+  int32_t* n_path;        /* [B]                                                      */
+  int32_t* next_token;    /* [B]                                                      */
+} falcon_accept_args;
+
+int falcon_tree_accept(falcon_ctx* ctx, const falcon_accept_args* args, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * falcon_kv_compact - keep the accepted path's K/V (Section 3.4: "record the
+ * accepted tokens and their corresponding features for the subsequent drafting
+ * phase", in its KV-cache form), all layers in one launch.
+ *
+ *   cache row L_b + j  <-  tree row path[b][j],   j = 0 .. n_path[b]-1
+ *   new_len[b] = L_b + n_path[b]
+ * In place by default (tree row t is cache row L_b + t; a destination row may be
+ * an earlier source row, which the kernel handles); with k/v_tree_layers the tree
+ * rows come from separate [N, Hkv, D] buffers.  Rows below L_b are untouched;
+ * rows at and above new_len[b] are unspecified afterwards.  prefix_len is not
+ * modified.
+ * ------------------------------------------------------------------------- */
+typedef struct {
+  falcon_tree_desc tree;  /* token unused                                             */
+  int32_t n_layers, n_kv_heads, head_dim;
+  void* const* k_cache_layers; /* device array [n_layers] of cache base pointers      */
+  void* const* v_cache_layers;
+  int64_t kv_stride_b, kv_stride_h, kv_stride_s;
+  int32_t s_cap;
+  const void* const* k_tree_layers; /* optional device array [n_layers]               */
+  const void* const* v_tree_layers;
+  const int32_t* path;    /* [B, path_stride] from falcon_tree_accept                 */
+  int32_t path_stride;
+  const int32_t* n_path;  /* [B]                                                      */
+  int32_t* new_len;       /* [B]                                                      */
+} falcon_compact_args;
+
+int falcon_kv_compact(falcon_ctx* ctx, const falcon_compact_args* args, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FALCON_H_ */

@@ -1,0 +1,167 @@
+// C-ABI entry points: argument validation, context management, dispatch.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+namespace falcon {
+
+int cuda_fail(falcon_ctx* ctx, cudaError_t e, const char* where) {
+  if (ctx) ctx->last_error = std::string(where) + ": " + cudaGetErrorString(e);
+  return FALCON_ERR_CUDA;
+}
+
+int ensure_workspace(falcon_ctx* ctx, size_t bytes) {
+  if (bytes <= ctx->ws_bytes) return FALCON_OK;
+  // cudaFree waits for work in flight, so a kernel still reading the old block is safe.
+  if (ctx->ws) cudaFree(ctx->ws);
+  ctx->ws = nullptr;
+  ctx->ws_bytes = 0;
+  const size_t want = bytes + bytes / 4;
+  cudaError_t e = cudaMalloc(&ctx->ws, want);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMalloc(workspace)");
+  ctx->ws_bytes = want;
+  return FALCON_OK;
+}
+
+int ensure_tickets(falcon_ctx* ctx, size_t count) {
+  if (count <= ctx->n_tickets) return FALCON_OK;
+  if (ctx->tickets) cudaFree(ctx->tickets);
+  ctx->tickets = nullptr;
+  ctx->n_tickets = 0;
+  const size_t want = count * 2 + 64;
+  cudaError_t e = cudaMalloc(&ctx->tickets, want * sizeof(int));
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMalloc(tickets)");
+  e = cudaMemset(ctx->tickets, 0, want * sizeof(int));
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMemset(tickets)");
+  ctx->n_tickets = want;
+  return FALCON_OK;
+}
+
+int check_tree_desc(const falcon_tree_desc& t, bool need_token) {
+  if (t.batch < 1 || t.total_nodes < t.batch || t.max_tree < 1 || t.max_prefix_len < 0) return FALCON_ERR_INVALID_ARG;
+  if (t.max_tree > FALCON_T_MAX) return FALCON_ERR_UNSUPPORTED;
+  if (!t.node_off || !t.parent || !t.prefix_len) return FALCON_ERR_INVALID_ARG;
+  if (need_token && !t.token) return FALCON_ERR_INVALID_ARG;
+  if (static_cast<int64_t>(t.max_tree) * t.batch < t.total_nodes) return FALCON_ERR_INVALID_ARG;
+  return FALCON_OK;
+}
+
+}  // namespace falcon
+
+using namespace falcon;
+
+extern "C" {
+
+int falcon_create(falcon_ctx** out, int device) {
+  if (!out) return FALCON_ERR_INVALID_ARG;
+  *out = nullptr;
+  cudaError_t e = cudaSetDevice(device);
+  if (e != cudaSuccess) return FALCON_ERR_CUDA;
+  cudaDeviceProp prop;
+  e = cudaGetDeviceProperties(&prop, device);
+  if (e != cudaSuccess) return FALCON_ERR_CUDA;
+  if (prop.major != 10) return FALCON_ERR_UNSUPPORTED;  // built for sm_100a only
+  falcon_ctx* ctx = new (std::nothrow) falcon_ctx();
+  if (!ctx) return FALCON_ERR_INVALID_ARG;
+  ctx->device = device;
+  ctx->sm_count = prop.multiProcessorCount;
+  ctx->smem_optin = static_cast<int>(prop.sharedMemPerBlockOptin);
+  *out = ctx;
+  return FALCON_OK;
+}
+
+int falcon_destroy(falcon_ctx* ctx) {
+  if (!ctx) return FALCON_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  tree_attn_tc_release(ctx);
+  if (ctx->ws) cudaFree(ctx->ws);
+  if (ctx->tickets) cudaFree(ctx->tickets);
+  delete ctx;
+  return FALCON_OK;
+}
+
+const char* falcon_status_string(int status) {
+  switch (status) {
+    case FALCON_OK: return "ok";
+    case FALCON_ERR_INVALID_ARG: return "invalid argument";
+    case FALCON_ERR_UNSUPPORTED: return "unsupported shape or device";
+    case FALCON_ERR_CUDA: return "CUDA error";
+    case FALCON_ERR_BAD_TREE: return "malformed tree";
+    case FALCON_ERR_CAPACITY: return "size exceeds capacity";
+    case FALCON_ERR_TIMEOUT: return "device wait timed out";
+    default: return "unknown status";
+  }
+}
+
+const char* falcon_last_error(const falcon_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
+
+int falcon_tree_validate_host(const int32_t* parent, int32_t T) {
+  if (!parent) return FALCON_ERR_INVALID_ARG;
+  if (T < 1) return FALCON_ERR_BAD_TREE;
+  if (T > FALCON_T_MAX) return FALCON_ERR_UNSUPPORTED;
+  if (parent[0] != -1) return FALCON_ERR_BAD_TREE;
+  for (int32_t i = 1; i < T; ++i)
+    if (parent[i] < 0 || parent[i] >= i) return FALCON_ERR_BAD_TREE;
+  return FALCON_OK;
+}
+
+int falcon_tree_attn(falcon_ctx* ctx, const falcon_attn_args* a, void* stream) {
+  if (!ctx || !a) return FALCON_ERR_INVALID_ARG;
+  int rc = check_tree_desc(a->tree, false);
+  if (rc) return rc;
+  if (!a->q || !a->out || !a->k_cache || !a->v_cache) return FALCON_ERR_INVALID_ARG;
+  if ((a->k_tree == nullptr) != (a->v_tree == nullptr)) return FALCON_ERR_INVALID_ARG;
+  if (a->n_q_heads < 1 || a->n_kv_heads < 1 || a->s_cap < 1) return FALCON_ERR_INVALID_ARG;
+  if (a->n_q_heads % a->n_kv_heads != 0) return FALCON_ERR_UNSUPPORTED;
+  if (a->head_dim != 64 && a->head_dim != 128) return FALCON_ERR_UNSUPPORTED;
+  if (a->kv_stride_s < a->head_dim || a->kv_stride_h < 0 || a->kv_stride_b < 0) return FALCON_ERR_INVALID_ARG;
+  if ((a->kv_stride_s | a->kv_stride_h | a->kv_stride_b) & 7) return FALCON_ERR_INVALID_ARG;
+  const uintptr_t align = reinterpret_cast<uintptr_t>(a->q) | reinterpret_cast<uintptr_t>(a->out) |
+                          reinterpret_cast<uintptr_t>(a->k_cache) | reinterpret_cast<uintptr_t>(a->v_cache) |
+                          reinterpret_cast<uintptr_t>(a->k_tree) | reinterpret_cast<uintptr_t>(a->v_tree);
+  if (align & 15) return FALCON_ERR_INVALID_ARG;
+  if (a->n_splits < 0 || a->n_splits > 64) return FALCON_ERR_INVALID_ARG;
+  if (!(a->sm_scale == a->sm_scale)) return FALCON_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  switch (a->kernel) {
+    case FALCON_ATTN_SIMT:
+      return launch_tree_attn_simt(ctx, *a, s);
+    case FALCON_ATTN_TC:
+      if (!tree_attn_tc_supports(ctx, *a)) return FALCON_ERR_UNSUPPORTED;
+      return launch_tree_attn_tc(ctx, *a, s);
+    case FALCON_ATTN_AUTO:
+      if (tree_attn_tc_supports(ctx, *a)) return launch_tree_attn_tc(ctx, *a, s);
+      return launch_tree_attn_simt(ctx, *a, s);
+    default:
+      return FALCON_ERR_INVALID_ARG;
+  }
+}
+
+int falcon_tree_accept(falcon_ctx* ctx, const falcon_accept_args* a, void* stream) {
+  if (!ctx || !a) return FALCON_ERR_INVALID_ARG;
+  int rc = check_tree_desc(a->tree, true);
+  if (rc) return rc;
+  if (!a->logits || !a->argmax_out || !a->path || !a->n_path || !a->next_token) return FALCON_ERR_INVALID_ARG;
+  if (a->vocab < 1 || a->logits_stride < a->vocab) return FALCON_ERR_INVALID_ARG;
+  if (a->path_stride < a->tree.max_tree) return FALCON_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(a->logits) & 3) return FALCON_ERR_INVALID_ARG;
+  return launch_tree_accept(ctx, *a, static_cast<cudaStream_t>(stream));
+}
+
+int falcon_kv_compact(falcon_ctx* ctx, const falcon_compact_args* a, void* stream) {
+  if (!ctx || !a) return FALCON_ERR_INVALID_ARG;
+  int rc = check_tree_desc(a->tree, false);
+  if (rc) return rc;
+  if (!a->k_cache_layers || !a->v_cache_layers || !a->path || !a->n_path || !a->new_len) return FALCON_ERR_INVALID_ARG;
+  if ((a->k_tree_layers == nullptr) != (a->v_tree_layers == nullptr)) return FALCON_ERR_INVALID_ARG;
+  if (a->n_layers < 1 || a->n_kv_heads < 1 || a->s_cap < 1) return FALCON_ERR_INVALID_ARG;
+  if (a->head_dim < 8 || a->head_dim > 256 || (a->head_dim & 7)) return FALCON_ERR_UNSUPPORTED;
+  if (a->kv_stride_s < a->head_dim || a->kv_stride_h < 0 || a->kv_stride_b < 0) return FALCON_ERR_INVALID_ARG;
+  if ((a->kv_stride_s | a->kv_stride_h | a->kv_stride_b) & 7) return FALCON_ERR_INVALID_ARG;
+  if (a->path_stride < a->tree.max_tree) return FALCON_ERR_INVALID_ARG;
+  return launch_kv_compact(ctx, *a, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,126 @@
+// falcon_kv_compact: the accepted path's K/V rows become the contiguous tail of
+// the cache, every layer and both K and V in one launch.  One CTA owns all rows
+// of one (layer, K|V, sequence, KV head): it reads every source row into
+// registers, passes a barrier, then writes, so a destination row that is also an
+// earlier source row (in-place mode) cannot be clobbered before it is read.
+// Launch/latency-bound byte copy with 16-byte accesses.
+#include "common.cuh"
+
+namespace falcon {
+namespace {
+
+constexpr int kCompactThreads = 256;
+constexpr int kMaxChunksPerThread = 16;  // 128 rows x 32 chunks (D = 256) / 256 threads
+
+struct CompactParams {
+  int32_t batch, n_layers, n_kv_heads, head_dim, s_cap, path_stride;
+  int64_t stride_b, stride_h, stride_s;
+  const int32_t* node_off;
+  const int32_t* prefix_len;
+  int32_t* status;
+  void* const* k_layers;
+  void* const* v_layers;
+  const void* const* k_tree_layers;
+  const void* const* v_tree_layers;
+  const int32_t* path;
+  const int32_t* n_path;
+  int32_t* new_len;
+};
+
+__global__ void __launch_bounds__(kCompactThreads) kv_compact_kernel(const CompactParams p) {
+  __shared__ int s_path[FALCON_T_MAX];
+  __shared__ int s_bad;
+  const int h = blockIdx.x, b = blockIdx.y;
+  const int layer = blockIdx.z >> 1, is_v = blockIdx.z & 1;
+  const int tid = threadIdx.x;
+
+  const int base = p.node_off[b];
+  const int T = p.node_off[b + 1] - base;
+  const int L = p.prefix_len[b];
+  const int n = p.n_path[b];
+  const bool separate = (p.k_tree_layers != nullptr);
+  int fault = 0;
+  if (T < 1 || T > FALCON_T_MAX || n < 1 || n > T) fault |= FALCON_DEV_BAD_PATH;
+  if (L < 0 || L + (separate ? n : T) > p.s_cap) fault |= FALCON_DEV_CAPACITY;
+  if (tid == 0) s_bad = 0;
+  __syncthreads();
+  if (!fault && tid < n) {
+    const int t = p.path[static_cast<int64_t>(b) * p.path_stride + tid];
+    s_path[tid] = t;
+    if (t < 0 || t >= T) s_bad = 1;
+  }
+  __syncthreads();
+  if (s_bad) fault |= FALCON_DEV_BAD_PATH;
+  const bool first = (h == 0 && blockIdx.z == 0 && tid == 0);
+  if (fault) {  // leave the cache alone, report, keep the old length
+    if (first) {
+      dev_status_or(p.status, b, fault);
+      p.new_len[b] = L;
+    }
+    return;
+  }
+  if (first) p.new_len[b] = L + n;
+
+  __nv_bfloat16* cache = static_cast<__nv_bfloat16*>(is_v ? p.v_layers[layer] : p.k_layers[layer]) +
+                         b * p.stride_b + h * p.stride_h;
+  const __nv_bfloat16* tree = nullptr;
+  if (separate)
+    tree = static_cast<const __nv_bfloat16*>(is_v ? p.v_tree_layers[layer] : p.k_tree_layers[layer]);
+
+  const int cpr = p.head_dim >> 3;  // 16-byte chunks per row
+  const int total = n * cpr;
+  uint4 regs[kMaxChunksPerThread];
+#pragma unroll
+  for (int k = 0; k < kMaxChunksPerThread; ++k) {
+    const int idx = tid + k * kCompactThreads;
+    if (idx < total) {
+      const int j = idx / cpr, c = idx - j * cpr;
+      const __nv_bfloat16* src =
+          separate ? tree + (static_cast<int64_t>(base + s_path[j]) * p.n_kv_heads + h) * p.head_dim
+                   : cache + static_cast<int64_t>(L + s_path[j]) * p.stride_s;
+      regs[k] = *reinterpret_cast<const uint4*>(src + 8 * c);
+    }
+  }
+  __syncthreads();  // every source row is in registers before any destination row is written
+#pragma unroll
+  for (int k = 0; k < kMaxChunksPerThread; ++k) {
+    const int idx = tid + k * kCompactThreads;
+    if (idx < total) {
+      const int j = idx / cpr, c = idx - j * cpr;
+      *reinterpret_cast<uint4*>(cache + static_cast<int64_t>(L + j) * p.stride_s + 8 * c) = regs[k];
+    }
+  }
+}
+
+}  // namespace
+
+int launch_kv_compact(falcon_ctx* ctx, const falcon_compact_args& a, cudaStream_t s) {
+  if (a.tree.batch > 65535 || 2 * static_cast<int64_t>(a.n_layers) > 65535) return FALCON_ERR_CAPACITY;
+  CompactParams p;
+  p.batch = a.tree.batch;
+  p.n_layers = a.n_layers;
+  p.n_kv_heads = a.n_kv_heads;
+  p.head_dim = a.head_dim;
+  p.s_cap = a.s_cap;
+  p.path_stride = a.path_stride;
+  p.stride_b = a.kv_stride_b;
+  p.stride_h = a.kv_stride_h;
+  p.stride_s = a.kv_stride_s;
+  p.node_off = a.tree.node_off;
+  p.prefix_len = a.tree.prefix_len;
+  p.status = a.tree.status;
+  p.k_layers = a.k_cache_layers;
+  p.v_layers = a.v_cache_layers;
+  p.k_tree_layers = a.k_tree_layers;
+  p.v_tree_layers = a.v_tree_layers;
+  p.path = a.path;
+  p.n_path = a.n_path;
+  p.new_len = a.new_len;
+  dim3 grid(a.n_kv_heads, a.tree.batch, 2 * a.n_layers);
+  kv_compact_kernel<<<grid, kCompactThreads, 0, s>>>(p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "kv_compact_kernel launch");
+  return FALCON_OK;
+}
+
+}  // namespace falcon
