@@ -1,0 +1,471 @@
+"""GPU parity: the CUDA library, called through the C ABI, against the CPU oracle
+on the same seeded inputs.  Integer outputs and caches are compared bit for bit;
+attention within max-abs 2e-2 and per-(sequence, head) relative L2 1e-2."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2412_12639_b200 import binding, synth
+
+import gpu_harness as H
+
+pytestmark = pytest.mark.gpu
+
+KERNELS = [binding.ATTN_SIMT, binding.ATTN_TC]
+
+
+def tc_or_skip(rc):
+    if rc == binding.ERR_UNSUPPORTED:
+        pytest.skip("shape not taken by the tensor-core kernel")
+    assert rc == binding.OK
+
+
+def strides_of(a):
+    return tuple(s // 2 for s in a.strides[:3])
+
+
+def oracle_attn(tb, Hq, Hkv, D, q, k, v, scale=None, **kw):
+    scale = 1.0 / math.sqrt(D) if scale is None else scale
+    return oracle.tree_attn(tb.node_off, tb.parent, tb.prefix_len, Hq, Hkv, D, scale, q, k, v, strides_of(k), **kw)
+
+
+def random_case(rng, sizes, prefs, Hq, Hkv, D, slack=0):
+    tb = H.make_trees(sizes, prefs, rng)
+    s_cap = int(max(p + t for p, t in zip(prefs, sizes))) + slack
+    q = synth.normal_bf16(rng, (tb.total_nodes, Hq, D))
+    k = synth.normal_bf16(rng, (tb.batch, Hkv, s_cap, D))
+    v = synth.normal_bf16(rng, (tb.batch, Hkv, s_cap, D))
+    return tb, q, k, v
+
+
+# ------------------------------------------------------------------ attention
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_attn_tiny_config(kernel):
+    spec = synth.SPECS["tiny"]
+    tb = synth.make_trees(spec)
+    q, k, v = synth.make_layer_qkv(spec, tb, 0)
+    ref = oracle_attn(tb, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, q, k, v)
+    out, rc = H.run_attn(H.DevTrees(tb), spec.n_q_heads, spec.n_kv_heads, spec.head_dim, q, k, v, kernel=kernel,
+                         check=False)
+    tc_or_skip(rc)
+    H.assert_attn_close(out, ref, tb.node_off)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("G", [1, 2, 4, 8])
+def test_attn_sweep_shapes(kernel, D, G):
+    rng = np.random.default_rng(1000 * D + G)
+    Hkv = 2
+    for T, L in [(1, 0), (1, 1), (2, 31), (15, 32), (33, 33), (60, 127), (64, 128), (65, 129), (128, 200),
+                 (97, 333), (128, 0)]:
+        tb, q, k, v = random_case(rng, [T], [L], Hkv * G, Hkv, D, slack=int(rng.integers(0, 5)))
+        ref = oracle_attn(tb, Hkv * G, Hkv, D, q, k, v)
+        out, rc = H.run_attn(H.DevTrees(tb), Hkv * G, Hkv, D, q, k, v, kernel=kernel, check=False)
+        tc_or_skip(rc)
+        H.assert_attn_close(out, ref, tb.node_off)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_attn_split_invariance_and_determinism(kernel):
+    rng = np.random.default_rng(7)
+    tb, q, k, v = random_case(rng, [60], [1024], 4, 4, 128)
+    ref = oracle_attn(tb, 4, 4, 128, q, k, v)
+    dt = H.DevTrees(tb)
+    outs = []
+    for splits in (1, 2, 3, 8):
+        out, rc = H.run_attn(dt, 4, 4, 128, q, k, v, kernel=kernel, n_splits=splits, check=False)
+        tc_or_skip(rc)
+        H.assert_attn_close(out, ref, tb.node_off)
+        out2, _ = H.run_attn(dt, 4, 4, 128, q, k, v, kernel=kernel, n_splits=splits)
+        np.testing.assert_array_equal(out, out2)       # same launch twice: bit-identical
+        outs.append(out)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_attn_ragged_batch_small(kernel):
+    rng = np.random.default_rng(21)
+    sizes = [20, 80, 1, 47, 64, 33]
+    prefs = [256, 40, 700, 0, 513, 129]
+    tb, q, k, v = random_case(rng, sizes, prefs, 4, 2, 128, slack=3)
+    ref = oracle_attn(tb, 4, 2, 128, q, k, v)
+    out, rc = H.run_attn(H.DevTrees(tb), 4, 2, 128, q, k, v, kernel=kernel, check=False)
+    tc_or_skip(rc)
+    H.assert_attn_close(out, ref, tb.node_off)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_attn_chain_star_and_wide_root(kernel):
+    rng = np.random.default_rng(5)
+    for parent in (synth.chain_tree(40), synth.star_tree(21), synth.chain_tree(128), synth.star_tree(128)):
+        T = len(parent)
+        tb = H.make_trees([T], [77], rng, parents=[parent])
+        q = synth.normal_bf16(rng, (T, 2, 128))
+        k = synth.normal_bf16(rng, (1, 2, 77 + T, 128))
+        v = synth.normal_bf16(rng, (1, 2, 77 + T, 128))
+        ref = oracle_attn(tb, 2, 2, 128, q, k, v)
+        out, rc = H.run_attn(H.DevTrees(tb), 2, 2, 128, q, k, v, kernel=kernel, check=False)
+        tc_or_skip(rc)
+        H.assert_attn_close(out, ref, tb.node_off)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_attn_ignores_rows_past_the_tree_even_if_nan(kernel):
+    rng = np.random.default_rng(6)
+    tb, q, k, v = random_case(rng, [30, 17], [100, 60], 2, 2, 128, slack=40)
+    for b in range(2):
+        end = tb.prefix_len[b] + tb.tree_size(b)
+        k[b, :, end:] = 0x7FC0      # NaN
+        v[b, :, end:] = 0x7F80      # +inf
+    ref = oracle_attn(tb, 2, 2, 128, q, k, v)
+    out, rc = H.run_attn(H.DevTrees(tb), 2, 2, 128, q, k, v, kernel=kernel, check=False)
+    tc_or_skip(rc)
+    H.assert_attn_close(out, ref, tb.node_off)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_attn_large_scores_do_not_overflow(kernel):
+    # keys whose scores grow along the sequence, with a big scale: the running maximum keeps moving up
+    rng = np.random.default_rng(8)
+    T, L, D = 24, 300, 128
+    tb = H.make_trees([T], [L], rng)
+    q = synth.f32_to_bf16_bits(np.ones((T, 1, D), np.float32))
+    ramp = np.linspace(-2.0, 2.0, L + T, dtype=np.float32)[None, None, :, None]
+    k = synth.f32_to_bf16_bits(np.broadcast_to(ramp, (1, 1, L + T, D)).copy())
+    v = synth.normal_bf16(rng, (1, 1, L + T, D))
+    ref = oracle_attn(tb, 1, 1, D, q, k, v, scale=1.0)
+    out, rc = H.run_attn(H.DevTrees(tb), 1, 1, D, q, k, v, scale=1.0, kernel=kernel, check=False)
+    tc_or_skip(rc)
+    H.assert_attn_close(out, ref, tb.node_off)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_attn_separate_tree_buffers(kernel):
+    rng = np.random.default_rng(9)
+    sizes, prefs = [40, 9], [130, 0]
+    tb, q, k, v = random_case(rng, sizes, prefs, 4, 2, 128)
+    kt = np.empty((tb.total_nodes, 2, 128), np.uint16)
+    vt = np.empty_like(kt)
+    k2, v2 = k.copy(), v.copy()
+    for b in range(2):
+        L, T, o = prefs[b], sizes[b], tb.node_off[b]
+        kt[o:o + T] = k[b, :, L:L + T].transpose(1, 0, 2)
+        vt[o:o + T] = v[b, :, L:L + T].transpose(1, 0, 2)
+        k2[b, :, L:] = 0x7FC0
+        v2[b, :, L:] = 0x7FC0
+    ref = oracle_attn(tb, 4, 2, 128, q, k, v)
+    out, rc = H.run_attn(H.DevTrees(tb), 4, 2, 128, q, k2, v2, k_tree=kt, v_tree=vt, kernel=kernel, check=False)
+    tc_or_skip(rc)
+    H.assert_attn_close(out, ref, tb.node_off)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_attn_caller_mask_rows(kernel):
+    # relaxed causal mask of the drafter (Section 3.4): ancestors plus the nodes of the same k-block
+    rng = np.random.default_rng(10)
+    T, L = 50, 90
+    tb, q, k, v = random_case(rng, [T], [L], 2, 2, 128)
+    rows = np.zeros((T, 2), np.uint64)
+    for i in range(T):
+        for a in oracle.ancestors(tb.parent, i):
+            rows[i, a >> 6] |= np.uint64(1) << np.uint64(a & 63)
+        mate = i ^ 1                                    # k = 2 blocks: (0,1), (2,3), ...
+        if mate < T:
+            rows[i, mate >> 6] |= np.uint64(1) << np.uint64(mate & 63)
+    ref = oracle_attn(tb, 2, 2, 128, q, k, v, tree_mask=rows)
+    out, rc = H.run_attn(H.DevTrees(tb), 2, 2, 128, q, k, v, tree_mask=rows, kernel=kernel, check=False)
+    tc_or_skip(rc)
+    H.assert_attn_close(out, ref, tb.node_off)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_attn_strided_cache_view(kernel):
+    # K and V interleaved in one allocation: [B, Hkv, s_cap, 2, D] -> row stride 2*D
+    rng = np.random.default_rng(12)
+    T, L, D = 33, 140, 128
+    tb = H.make_trees([T], [L], rng)
+    q = synth.normal_bf16(rng, (T, 2, D))
+    kv = synth.normal_bf16(rng, (1, 2, L + T, 2, D))
+    k, v = kv[:, :, :, 0], kv[:, :, :, 1]
+    ref = oracle.tree_attn(tb.node_off, tb.parent, tb.prefix_len, 2, 2, D, 1 / math.sqrt(D), q, k, v, strides_of(k))
+    kvd = H.dev_bf16(kv)
+    qd = H.dev_bf16(q)
+    out = torch.zeros_like(qd)
+    dt = H.DevTrees(tb)
+    kd, vd = kvd[:, :, :, 0], kvd[:, :, :, 1]
+    a = binding.attn_args(dt.desc(), 2, 2, D, 1 / math.sqrt(D), qd, out, kd.data_ptr(), vd.data_ptr(),
+                          tuple(int(s) for s in kd.stride()[:3]), L + T, kernel=kernel)
+    rc = H.ctx().falcon_tree_attn(a, check=False)
+    tc_or_skip(rc)
+    torch.cuda.synchronize()
+    H.assert_attn_close(H.host_bits(out), ref, tb.node_off)
+
+
+def test_attn_malformed_tree_and_capacity_set_status_without_faulting():
+    rng = np.random.default_rng(13)
+    tb, q, k, v = random_case(rng, [10, 12], [20, 30], 2, 2, 128)
+    tb.parent[3] = 7                      # parent after child in sequence 0
+    dt = H.DevTrees(tb)
+    for kernel in KERNELS:
+        dt.status.zero_()
+        out, rc = H.run_attn(dt, 2, 2, 128, q, k, v, kernel=kernel, check=False)
+        if rc == binding.ERR_UNSUPPORTED:
+            continue
+        st = dt.status.cpu().numpy()
+        assert st[0] & binding.DEV_BAD_TREE and st[1] == 0
+        # sequence 1 is well formed: its rows are still right
+        ref = oracle_attn(synth.TreeBatch(np.array([0, 12], np.int32), tb.parent[10:], tb.token[10:],
+                                          tb.prefix_len[1:], tb.p_accept[1:]), 2, 2, 128, q[10:], k[1:], v[1:])
+        H.assert_attn_close(out[10:], ref, np.array([0, 12]))
+    # tree rows that do not fit the cache
+    tb2, q, k, v = random_case(rng, [10], [20], 2, 2, 128)
+    dt2 = H.DevTrees(tb2)
+    for kernel in KERNELS:
+        dt2.status.zero_()
+        _, rc = H.run_attn(dt2, 2, 2, 128, q, k, v, s_cap=25, kernel=kernel, check=False)
+        if rc == binding.ERR_UNSUPPORTED:
+            continue
+        assert dt2.status.cpu().numpy()[0] & binding.DEV_CAPACITY
+
+
+FULL = {"v7b": [0, 17, 31], "l13b": [3, 22, 39], "l70b": [1, 5], "ragged": [2, 30]}
+
+
+@pytest.mark.parametrize("name", ["v7b", "l13b", "l70b", "ragged"])
+def test_attn_full_size_configs_sampled_heads(name):
+    """Full-size launch (the one the benchmark times); the oracle checks a sample of KV heads of one layer."""
+    spec = synth.SPECS[name]
+    tb = synth.make_trees(spec)
+    q, k, v = synth.make_layer_qkv(spec, tb, 1)
+    out, _ = H.run_attn(H.DevTrees(tb), spec.n_q_heads, spec.n_kv_heads, spec.head_dim, q, k, v)
+    G = spec.n_q_heads // spec.n_kv_heads
+    for kvh in [h % spec.n_kv_heads for h in FULL[name]]:
+        qs = np.ascontiguousarray(q[:, kvh * G:(kvh + 1) * G])
+        ks = np.ascontiguousarray(k[:, kvh:kvh + 1])
+        vs = np.ascontiguousarray(v[:, kvh:kvh + 1])
+        ref = oracle_attn(tb, G, 1, spec.head_dim, qs, ks, vs)
+        H.assert_attn_close(np.ascontiguousarray(out[:, kvh * G:(kvh + 1) * G]), ref, tb.node_off)
+
+
+# --------------------------------------------------------------------- accept
+@pytest.mark.parametrize("name", ["tiny", "v7b", "l13b", "l70b", "ragged"])
+def test_accept_configs_bit_exact(name):
+    spec = synth.SPECS[name]
+    tb = synth.make_trees(spec)
+    logits = synth.make_logits(spec, tb)
+    g_ref = oracle.argmax(logits)
+    p_ref, n_ref, t_ref = oracle.tree_accept(tb.node_off, tb.parent, tb.token, g_ref)
+    g, path, n, nxt = H.run_accept(H.DevTrees(tb), logits)
+    np.testing.assert_array_equal(g, g_ref)
+    np.testing.assert_array_equal(n, n_ref)
+    np.testing.assert_array_equal(path, p_ref)
+    np.testing.assert_array_equal(nxt, t_ref)
+    # a second call on the same context gives the same result (arrival counters were reset)
+    g2, path2, n2, nxt2 = H.run_accept(H.DevTrees(tb), logits)
+    np.testing.assert_array_equal(path2, p_ref)
+    np.testing.assert_array_equal(g2, g_ref)
+
+
+@pytest.mark.parametrize("V,stride", [(1, 1), (3, 5), (1000, 1000), (4099, 4101), (32001, 32001), (32000, 32004),
+                                      (50000, 50001)])
+def test_accept_argmax_odd_vocab_and_strides(V, stride):
+    rng = np.random.default_rng(V)
+    tb = H.make_trees([37, 5], [0, 0], rng, vocab=max(1, min(V, 50)))
+    logits = rng.standard_normal((42, stride)).astype(np.float32)
+    logits[:, V:] = 100.0                              # padding columns must be ignored
+    g_ref = oracle.argmax(logits, vocab=V)
+    p_ref, n_ref, t_ref = oracle.tree_accept(tb.node_off, tb.parent, tb.token, g_ref)
+    g, path, n, nxt = H.run_accept(H.DevTrees(tb), logits, vocab=V)
+    np.testing.assert_array_equal(g, g_ref)
+    np.testing.assert_array_equal(path, p_ref)
+    np.testing.assert_array_equal(n, n_ref)
+    np.testing.assert_array_equal(nxt, t_ref)
+
+
+def test_accept_argmax_ties_nan_inf_and_signed_zero():
+    rng = np.random.default_rng(3)
+    V = 9000
+    tb = H.make_trees([8], [0], rng)
+    x = rng.standard_normal((8, V)).astype(np.float32)
+    x[0, [100, 5000, 8999]] = 77.0                     # ties far apart (different chunks): lowest index
+    x[1] = np.nan
+    x[2] = -np.inf
+    x[3] = 0.0
+    x[3, ::2] = -0.0
+    x[4, :4000] = np.nan
+    x[4, 4000:] = -np.inf                              # nothing above -inf: 0
+    x[5, 17] = np.inf
+    x[5, 16] = np.nan
+    x[6, :] = -np.inf
+    x[6, 8191] = -3.0
+    x[7, 0] = np.nan
+    x[7, 1:] = -np.inf
+    g_ref = oracle.argmax(x)
+    assert g_ref.tolist()[:8] == [100, 0, 0, 0, 0, 17, 8191, 0]
+    g, _, _, _ = H.run_accept(H.DevTrees(tb), x)
+    np.testing.assert_array_equal(g, g_ref)
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_accept_random_trees_small_vocab_bit_exact(seed):
+    rng = np.random.default_rng(seed)
+    sizes = [int(rng.integers(1, 129)) for _ in range(16)]
+    tb = H.make_trees(sizes, [0] * 16, rng, vocab=5)
+    logits = rng.standard_normal((tb.total_nodes, 5)).astype(np.float32)
+    g_ref = oracle.argmax(logits)
+    p_ref, n_ref, t_ref = oracle.tree_accept(tb.node_off, tb.parent, tb.token, g_ref)
+    g, path, n, nxt = H.run_accept(H.DevTrees(tb), logits)
+    np.testing.assert_array_equal(g, g_ref)
+    np.testing.assert_array_equal(path, p_ref)
+    np.testing.assert_array_equal(n, n_ref)
+    np.testing.assert_array_equal(nxt, t_ref)
+
+
+def test_accept_malformed_tree_reports_and_returns_root():
+    rng = np.random.default_rng(2)
+    tb = H.make_trees([6, 6], [0, 0], rng, vocab=4)
+    tb.parent[8] = 5                                   # sequence 1: parent[2] = 5 >= 2
+    logits = rng.standard_normal((12, 4)).astype(np.float32)
+    dt = H.DevTrees(tb)
+    g, path, n, nxt = H.run_accept(dt, logits)
+    st = dt.status.cpu().numpy()
+    assert st[0] == 0 and st[1] & binding.DEV_BAD_TREE
+    assert n[1] == 1 and path[1, 0] == 0 and nxt[1] == g[6]
+
+
+# -------------------------------------------------------------------- compact
+def accepted_paths(tb, rng, force=None):
+    B = tb.batch
+    path = np.full((B, 128), -1, np.int32)
+    n_path = np.zeros(B, np.int32)
+    for b in range(B):
+        par = tb.parent[tb.node_off[b]:tb.node_off[b + 1]]
+        node = int(rng.integers(0, len(par))) if force is None else force[b]
+        chain = oracle.ancestors(par, node)[::-1]
+        path[b, :len(chain)] = chain
+        n_path[b] = len(chain)
+    return path, n_path
+
+
+def check_compact(tb, Hkv, D, n_layers, rng, path, n_path, separate=False, slack=2):
+    s_cap = int((tb.prefix_len + np.diff(tb.node_off)).max()) + slack
+    ks = [rng.integers(0, 65536, size=(tb.batch, Hkv, s_cap, D)).astype(np.uint16) for _ in range(n_layers)]
+    vs = [rng.integers(0, 65536, size=(tb.batch, Hkv, s_cap, D)).astype(np.uint16) for _ in range(n_layers)]
+    kt = vt = None
+    if separate:
+        kt = [rng.integers(0, 65536, size=(tb.total_nodes, Hkv, D)).astype(np.uint16) for _ in range(n_layers)]
+        vt = [rng.integers(0, 65536, size=(tb.total_nodes, Hkv, D)).astype(np.uint16) for _ in range(n_layers)]
+    gk, gv, new_len = H.run_compact(H.DevTrees(tb), Hkv, D, ks, vs, path, n_path, kt, vt)
+    for l in range(n_layers):
+        for ref, got, tree in ((ks[l], gk[l], kt), (vs[l], gv[l], vt)):
+            before = ref.copy()
+            nl = oracle.kv_compact(tb.node_off, tb.prefix_len, Hkv, D, ref, strides_of(ref), s_cap, path, n_path,
+                                   tree_rows=None if tree is None else (kt[l] if ref is ks[l] else vt[l]))
+            np.testing.assert_array_equal(new_len, nl)
+            for b in range(tb.batch):
+                np.testing.assert_array_equal(got[b, :, :nl[b]], ref[b, :, :nl[b]])
+                np.testing.assert_array_equal(got[b, :, :tb.prefix_len[b]], before[b, :, :tb.prefix_len[b]])
+
+
+@pytest.mark.parametrize("name,layers", [("tiny", 1), ("v7b", 3), ("l13b", 2), ("l70b", 3), ("ragged", 2)])
+def test_compact_configs_bit_exact_with_accepted_paths(name, layers):
+    spec = synth.SPECS[name]
+    tb = synth.make_trees(spec)
+    logits = synth.make_logits(spec, tb)
+    g = oracle.argmax(logits)
+    path, n_path, _ = oracle.tree_accept(tb.node_off, tb.parent, tb.token, g)
+    check_compact(tb, spec.n_kv_heads, spec.head_dim, layers, np.random.default_rng(0), path, n_path)
+
+
+@pytest.mark.parametrize("separate", [False, True])
+@pytest.mark.parametrize("D", [64, 128, 256])
+def test_compact_random_paths_overlap_and_identity(separate, D):
+    rng = np.random.default_rng(D + separate)
+    sizes = [128, 1, 40, 77]
+    parents = [synth.chain_tree(128), np.array([-1], np.int32), synth.random_shape_tree(rng, 40),
+               synth.random_shape_tree(rng, 77)]
+    tb = H.make_trees(sizes, [5, 0, 64, 300], rng, parents=parents)
+    # full chain of 128 (identity, the largest copy), single node, two random leaves
+    path, n_path = accepted_paths(tb, rng, force=[127, 0, 39, 76])
+    check_compact(tb, 3, D, 2, rng, path, n_path, separate=separate)
+    path, n_path = accepted_paths(tb, rng)
+    check_compact(tb, 3, D, 2, rng, path, n_path, separate=separate)
+
+
+def test_compact_handworked_overlap_path():
+    rng = np.random.default_rng(4)
+    tb = H.make_trees([4], [2], rng, parents=[np.array([-1, 0, 0, 2], np.int32)])
+    path = np.full((1, 128), -1, np.int32)
+    path[0, :3] = [0, 2, 3]
+    check_compact(tb, 2, 64, 1, rng, path, np.array([3], np.int32), slack=0)
+
+
+def test_compact_bad_path_or_capacity_leaves_cache_untouched():
+    rng = np.random.default_rng(5)
+    tb = H.make_trees([6, 6], [4, 4], rng)
+    path = np.full((2, 128), -1, np.int32)
+    path[:, 0] = 0
+    path[1, 1] = 9                                      # outside the tree
+    n_path = np.array([1, 2], np.int32)
+    s_cap = 12
+    ks = [rng.integers(0, 65536, size=(2, 2, s_cap, 64)).astype(np.uint16)]
+    vs = [rng.integers(0, 65536, size=(2, 2, s_cap, 64)).astype(np.uint16)]
+    dt = H.DevTrees(tb)
+    gk, gv, new_len = H.run_compact(dt, 2, 64, ks, vs, path, n_path)
+    st = dt.status.cpu().numpy()
+    assert st[0] == 0 and st[1] & binding.DEV_BAD_PATH
+    assert new_len.tolist() == [5, 4]
+    np.testing.assert_array_equal(gk[0][1], ks[0][1])
+    np.testing.assert_array_equal(gv[0][1], vs[0][1])
+
+
+# ------------------------------------------------------------------------ ABI
+def test_abi_rejects_bad_arguments_without_launching():
+    rng = np.random.default_rng(1)
+    tb, q, k, v = random_case(rng, [8], [16], 2, 2, 128)
+    dt = H.DevTrees(tb)
+    qd, kd, vd = H.dev_bf16(q), H.dev_bf16(k), H.dev_bf16(v)
+    out = torch.zeros_like(qd)
+    st = tuple(int(s) for s in kd.stride()[:3])
+    c = H.ctx()
+
+    def attn(**kw):
+        base = dict(tree=dt.desc(), n_q_heads=2, n_kv_heads=2, head_dim=128, sm_scale=0.1, q=qd, out=out, k_cache=kd,
+                    v_cache=vd, strides=st, s_cap=24)
+        base.update(kw)
+        return c.falcon_tree_attn(binding.attn_args(**base), check=False)
+
+    assert attn() == binding.OK
+    assert attn(q=None) == binding.ERR_INVALID_ARG
+    assert attn(head_dim=96) == binding.ERR_UNSUPPORTED
+    assert attn(n_q_heads=3) == binding.ERR_UNSUPPORTED
+    assert attn(strides=(st[0], st[1], 100)) == binding.ERR_INVALID_ARG
+    assert attn(q=qd.data_ptr() + 2) == binding.ERR_INVALID_ARG
+    assert attn(kernel=9) == binding.ERR_INVALID_ARG
+    assert attn(n_splits=65) == binding.ERR_INVALID_ARG
+    assert attn(k_tree=kd) == binding.ERR_INVALID_ARG          # k_tree without v_tree
+    big = dt.desc()
+    big.max_tree = 129
+    assert attn(tree=big) == binding.ERR_UNSUPPORTED
+    none = dt.desc()
+    none.parent = None
+    assert attn(tree=none) == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.FalconError):
+        c.falcon_tree_attn(binding.attn_args(dt.desc(), 2, 2, 96, 0.1, qd, out, kd, vd, st, 24))
+
+    lg = torch.zeros(8, 10, device="cuda")
+    i32 = lambda *s: torch.zeros(*s, dtype=torch.int32, device="cuda")
+    g, path, n, nxt = i32(8), i32(1, 128), i32(1), i32(1)
+    assert c.falcon_tree_accept(binding.accept_args(dt.desc(), 10, lg, 10, g, path, 128, n, nxt), check=False) == 0
+    assert c.falcon_tree_accept(binding.accept_args(dt.desc(), 10, lg, 9, g, path, 128, n, nxt), check=False) \
+        == binding.ERR_INVALID_ARG
+    assert c.falcon_tree_accept(binding.accept_args(dt.desc(), 0, lg, 10, g, path, 128, n, nxt), check=False) \
+        == binding.ERR_INVALID_ARG
+    assert c.falcon_tree_accept(binding.accept_args(dt.desc(), 10, lg, 10, g, path, 4, n, nxt), check=False) \
+        == binding.ERR_INVALID_ARG
+    assert c.falcon_tree_accept(binding.accept_args(dt.desc(), 10, None, 10, g, path, 128, n, nxt), check=False) \
+        == binding.ERR_INVALID_ARG
+    torch.cuda.synchronize()
