@@ -1,0 +1,395 @@
+"""Benchmark of the tree-verification step (n_layers x falcon_tree_attn +
+falcon_tree_accept + falcon_kv_compact) on synthetic Vicuna/LLaMA2-shaped inputs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload v7b] [--impl falcon|reference]
+
+Prints ONE JSON line.  `value` is whole-job verify steps/s with every input
+resident in HBM (the step replayed as CUDA graphs, device-timed with CUDA
+events); `e2e` is the same step driven from pinned host buffers with the
+host<->device copies inside the timed region; `roofline` is the attention
+kernel's algorithmic bytes per launch over its measured launch time;
+`cpu_baseline` is the CPU oracle timed on a bounded sample of the same workload.
+With --impl reference the oracle itself is the timed arm.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2412_12639_b200 import synth  # noqa: E402
+
+METRIC = "tree-verify steps/sec"
+UNIT = "steps/s"
+
+
+# --------------------------------------------------------------------------- bytes
+def attn_bytes_per_layer(spec, tb) -> int:
+    """Algorithmic bytes of one attention launch: K and V rows of prefix+tree once, q read, out written."""
+    total = 0
+    for b in range(tb.batch):
+        L, T = int(tb.prefix_len[b]), tb.tree_size(b)
+        total += 2 * spec.n_kv_heads * (L + T) * spec.head_dim * 2 + 2 * T * spec.n_q_heads * spec.head_dim * 2 + 4 * T
+    return total
+
+
+def accept_bytes(spec, tb) -> int:
+    return 4 * tb.total_nodes * spec.vocab + 12 * tb.total_nodes
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx = float(f[1])
+            except ValueError:
+                continue
+            for n, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- oracle timing (CPU)
+def time_oracle_step(spec, tb, logits, sample_layers: int):
+    """Runs the CPU oracle on `sample_layers` layers of attention and compaction plus the full acceptance,
+    and extrapolates one whole step.  Returns (seconds per step, threads, description)."""
+    import oracle
+    scale = 1.0 / math.sqrt(spec.head_dim)
+    t_attn = t_comp = 0.0
+    g = oracle.argmax(logits)
+    path, n_path, _ = oracle.tree_accept(tb.node_off, tb.parent, tb.token, g)
+    for layer in range(sample_layers):
+        q, k, v = synth.make_layer_qkv(spec, tb, layer)
+        st = tuple(s // 2 for s in k.strides[:3])
+        t0 = time.perf_counter()
+        oracle.tree_attn(tb.node_off, tb.parent, tb.prefix_len, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, scale,
+                         q, k, v, st)
+        t1 = time.perf_counter()
+        oracle.kv_compact(tb.node_off, tb.prefix_len, spec.n_kv_heads, spec.head_dim, k, st, k.shape[2], path, n_path)
+        oracle.kv_compact(tb.node_off, tb.prefix_len, spec.n_kv_heads, spec.head_dim, v, st, v.shape[2], path, n_path)
+        t2 = time.perf_counter()
+        t_attn += t1 - t0
+        t_comp += t2 - t1
+    t0 = time.perf_counter()
+    g = oracle.argmax(logits)
+    oracle.tree_accept(tb.node_off, tb.parent, tb.token, g)
+    t_acc = time.perf_counter() - t0
+    step = (t_attn + t_comp) / sample_layers * spec.n_layers + t_acc
+    desc = "%d of %d layers of attention+compaction and the full acceptance, extrapolated to one step" % (
+        sample_layers, spec.n_layers)
+    return step, oracle.max_threads(), desc
+
+
+def oracle_sample_layers(spec, tb) -> int:
+    # scalar double flops of one layer of attention; aim at roughly 10-20 s on a few cores
+    flops = 4.0 * spec.head_dim * spec.n_q_heads * sum(
+        tb.tree_size(b) * (int(tb.prefix_len[b]) + tb.tree_size(b)) for b in range(tb.batch))
+    return max(1, min(spec.n_layers, int(12e9 / max(flops, 1.0))))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    spec = synth.SPECS[args.workload]
+    tb = synth.make_trees(spec)
+    logits = synth.make_logits(spec, tb)
+    per_step_layers = max(1, oracle_sample_layers(spec, tb) // max(1, args.steps + args.warmup))
+    for _ in range(args.warmup):
+        time_oracle_step(spec, tb, logits, per_step_layers)
+    times, threads, desc = [], 1, ""
+    for _ in range(args.steps):
+        t, threads, desc = time_oracle_step(spec, tb, logits, per_step_layers)
+        times.append(t)
+    sec = sum(times) / len(times)
+    val = 1.0 / sec
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "note": "CPU oracle, host cores only"},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- GPU arm
+def run_falcon(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2412_12639_b200 as falcon
+    from paper_2412_12639_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    ctx = falcon.Context(local)
+
+    spec = synth.SPECS[args.workload]
+    # every rank verifies its own batch of sequences (independent problems: no exchange on this path)
+    tb = synth.make_trees(spec, seed=spec.seed + rank)
+    logits_h = synth.make_logits(spec, tb, seed=spec.seed + rank)
+    s_cap = synth.cache_capacity(tb)
+    B, N, Hq, Hkv, D, NL = tb.batch, tb.total_nodes, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.n_layers
+    scale = 1.0 / math.sqrt(D)
+
+    def i32(a):
+        return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+
+    node_off, parent, token, prefix = i32(tb.node_off), i32(tb.parent), i32(tb.token), i32(tb.prefix_len)
+    status = torch.zeros(B, dtype=torch.int32, device=dev)
+    tree = binding.tree_desc(B, N, tb.max_tree, int(tb.prefix_len.max()), node_off, parent, prefix, token=token,
+                             status=status)
+
+    # all layers' caches in one allocation [NL, 2, B, Hkv, s_cap, D]; q and out [NL, N, Hq, D]
+    cache = torch.empty((NL, 2, B, Hkv, s_cap, D), dtype=torch.bfloat16, device=dev)
+    q_all = torch.empty((NL, N, Hq, D), dtype=torch.bfloat16, device=dev)
+    out_all = torch.zeros_like(q_all)
+    q_host = torch.empty((NL, N, Hq, D), dtype=torch.bfloat16).pin_memory()
+    # the tree's own K/V rows of every layer, as the host hands them over each step (e2e leg)
+    tree_rows = [(b, int(tb.prefix_len[b]), tb.tree_size(b)) for b in range(B)]
+    tkv_host = [torch.empty((NL, 2, Hkv, T, D), dtype=torch.bfloat16).pin_memory() for (_, _, T) in tree_rows]
+    for layer in range(NL):
+        qh, kh, vh = synth.make_layer_qkv(spec, tb, layer, s_cap=s_cap, seed=spec.seed + rank)
+        q_host[layer] = torch.from_numpy(qh.view(np.int16)).view(torch.bfloat16)
+        kt = torch.from_numpy(kh.view(np.int16)).view(torch.bfloat16)
+        vt = torch.from_numpy(vh.view(np.int16)).view(torch.bfloat16)
+        cache[layer, 0].copy_(kt)
+        cache[layer, 1].copy_(vt)
+        for (b, L, T), th in zip(tree_rows, tkv_host):
+            th[layer, 0] = kt[b, :, L:L + T]
+            th[layer, 1] = vt[b, :, L:L + T]
+    q_all.copy_(q_host)
+    logits_host = torch.from_numpy(logits_h).pin_memory()
+    logits = logits_host.to(dev)
+    tree_host = torch.from_numpy(np.concatenate([tb.node_off, tb.parent, tb.token, tb.prefix_len]).astype(np.int32)
+                                 ).pin_memory()
+    tree_dev = torch.empty_like(tree_host, device=dev)
+
+    g = torch.zeros(N, dtype=torch.int32, device=dev)
+    path = torch.zeros((B, 128), dtype=torch.int32, device=dev)
+    n_path = torch.zeros(B, dtype=torch.int32, device=dev)
+    nxt = torch.zeros(B, dtype=torch.int32, device=dev)
+    new_len = torch.zeros(B, dtype=torch.int32, device=dev)
+    result_dev = torch.zeros(3 * B + B * 128, dtype=torch.int32, device=dev)
+    result_host = torch.zeros(3 * B + B * 128, dtype=torch.int32).pin_memory()
+    kptr = torch.tensor([cache[l, 0].data_ptr() for l in range(NL)], dtype=torch.int64, device=dev)
+    vptr = torch.tensor([cache[l, 1].data_ptr() for l in range(NL)], dtype=torch.int64, device=dev)
+    strides = tuple(int(s) for s in cache[0, 0].stride()[:3])
+
+    attn = [binding.attn_args(tree, Hq, Hkv, D, scale, q_all[l], out_all[l], cache[l, 0], cache[l, 1], strides, s_cap)
+            for l in range(NL)]
+    acc = binding.accept_args(tree, spec.vocab, logits, logits.shape[1], g, path, 128, n_path, nxt)
+    cmp_ = binding.compact_args(tree, NL, Hkv, D, kptr, vptr, strides, s_cap, path, 128, n_path, new_len)
+
+    def launch_attn():
+        for a in attn:
+            ctx.falcon_tree_attn(a)
+
+    def launch_tail():
+        ctx.falcon_tree_accept(acc)
+        ctx.falcon_kv_compact(cmp_)
+
+    stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        launch_attn()           # first calls allocate scratch: before any capture
+        launch_tail()
+        stream.synchronize()
+        g_attn, g_tail = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_attn, stream=stream):
+            launch_attn()
+        with torch.cuda.graph(g_tail, stream=stream):
+            launch_tail()
+
+        def barrier():
+            torch.cuda.synchronize()
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
+
+        # ---------------- device-resident steps ----------------
+        for _ in range(args.warmup):
+            g_attn.replay()
+            g_tail.replay()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+        sampler = ClockSampler(local)
+        barrier()
+        sampler.start()
+        t_wall = time.perf_counter()
+        for s in range(args.steps):
+            ev[s][0].record(stream)
+            g_attn.replay()
+            ev[s][1].record(stream)
+            g_tail.replay()
+            ev[s][2].record(stream)
+        barrier()
+        t_wall = time.perf_counter() - t_wall
+        total_ms = ev[0][0].elapsed_time(ev[-1][2])
+        attn_ms = sum(e[0].elapsed_time(e[1]) for e in ev)
+
+        # ---------------- end to end from pinned host buffers ----------------
+        def e2e_step():
+            tree_dev.copy_(tree_host, non_blocking=True)
+            q_all.copy_(q_host, non_blocking=True)
+            for (b, L, T), th in zip(tree_rows, tkv_host):
+                cache[:, :, b, :, L:L + T].copy_(th, non_blocking=True)
+            logits.copy_(logits_host, non_blocking=True)
+            g_attn.replay()
+            g_tail.replay()
+            result_dev[:B].copy_(n_path)
+            result_dev[B:2 * B].copy_(nxt)
+            result_dev[2 * B:3 * B].copy_(new_len)
+            result_dev[3 * B:].copy_(path.view(-1))
+            result_host.copy_(result_dev, non_blocking=True)
+            stream.synchronize()
+
+        for _ in range(max(1, min(args.warmup, 3))):
+            e2e_step()
+        e2e_steps = max(3, min(args.steps, 20))
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        clocks = sampler.stop()
+
+    if world > 1:
+        t = torch.tensor([total_ms, attn_ms, e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, attn_ms, e2e_ms = (float(x) for x in t.tolist())
+    if status.any().item():
+        raise RuntimeError("device status words set: %s" % status.tolist())
+
+    h2d = (tree_host.numel() * 4 + q_host.numel() * 2 + sum(t.numel() for t in tkv_host) * 2 + logits_host.numel() * 4)
+    d2h = result_host.numel() * 4
+    ms_per_step = total_ms / args.steps
+    per_launch_us = attn_ms / (args.steps * NL) * 1e3
+    a_bytes = attn_bytes_per_layer(spec, tb)
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except OSError:
+        pass
+    peak = float(peaks.get("hbm_gbs", 6650.0))
+    achieved = a_bytes / (per_launch_us * 1e-6) / 1e9
+    traffic = None
+    try:
+        traffic = json.load(open(os.path.join(ROOT, "profiles", "traffic.json"))).get(args.workload)
+    except (OSError, ValueError):
+        pass
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        sl = oracle_sample_layers(spec, tb)
+        sec, threads, desc = time_oracle_step(spec, tb, logits_h, sl)
+        cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+
+    step_bytes = NL * a_bytes + accept_bytes(spec, tb)
+    line = {
+        "metric": METRIC, "value": world * 1e3 / ms_per_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "batch": B, "n_layers": NL, "n_q_heads": Hq, "n_kv_heads": Hkv,
+                   "head_dim": D, "prefix_len": tb.prefix_len.tolist(), "tree_nodes": np.diff(tb.node_off).tolist(),
+                   "vocab": spec.vocab, "parallelism": "replicas x%d (independent sequences, no collective)" % world,
+                   "l2": "inputs larger than L2: %.0f MB of distinct K/V, q and logits per step" % (step_bytes / 1e6),
+                   "timing": "CUDA graphs replayed on one stream, CUDA events, max over ranks"},
+        "us_per_layer": per_launch_us,
+        "roofline": {"bound": "hbm", "kernel": "falcon_tree_attn", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": traffic, "bytes_per_launch": a_bytes,
+                     "us_per_launch": per_launch_us,
+                     "peak_source": "MEASURED_PEAKS.json hbm_gbs" if peaks else "fallback 6650 GB/s"},
+        "e2e": {"value": world * e2e_steps * 1e3 / e2e_ms, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h},
+        "gpu_launches": args.steps * (NL + 2),
+        "clocks": clocks,
+        "cpu_baseline": cpu,
+        "wall_s_timed": t_wall,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="v7b", choices=sorted(synth.SPECS))
+    ap.add_argument("--impl", default="falcon", choices=["falcon", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "falcon":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_falcon(args)
+
+
+if __name__ == "__main__":
+    main()
