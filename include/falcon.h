@@ -157,6 +157,33 @@ typedef struct {
 int falcon_tree_accept(falcon_ctx* ctx, const falcon_accept_args* args, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * falcon_tree_accept_static - falcon_tree_accept for callers that cannot allocate
+ * device memory.  (The paper has no counterpart: this is a deployment variant of
+ * the call above, same arguments, same results.)
+ *
+ * Who needs it: a serving process whose device memory is owned entirely by its
+ * own pool, a process pinned to a fixed memory budget, or a latency-critical
+ * loop that cannot risk the device-wide synchronisation an allocation can cause.
+ * This call needs no falcon_ctx and never calls cudaMalloc, cudaFree or any
+ * allocating routine.  Its scratch (argmax partials, arrival counters) is a fixed
+ * array inside the library image, about 0.5 MB, which every GPU that loads the
+ * library holds until the process exits.
+ *
+ * Limits: total_nodes <= FALCON_STATIC_MAX_NODES and batch <=
+ * FALCON_STATIC_MAX_BATCH; anything larger returns FALCON_ERR_CAPACITY and
+ * launches nothing.  It runs on the current device.  The first call on each
+ * device looks up the array's device address (a one-time set-up step); make that
+ * first call before any stream capture begins.  All calls on a device share the
+ * one array, and it keeps the previous call's contents: the call itself clears
+ * the counters it needs at zero, but two calls that overlap on the GPU (different
+ * streams, no ordering between them) race on it and give wrong results -
+ * serialise them.
+ * ------------------------------------------------------------------------- */
+#define FALCON_STATIC_MAX_NODES 1024
+#define FALCON_STATIC_MAX_BATCH 256
+int falcon_tree_accept_static(const falcon_accept_args* args, void* stream);
+
+/* ---------------------------------------------------------------------------
  * falcon_kv_compact - keep the accepted path's K/V (Section 3.4: "record the
  * accepted tokens and their corresponding features for the subsequent drafting
  * phase", in its KV-cache form), all layers in one launch.

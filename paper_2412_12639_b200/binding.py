@@ -83,6 +83,8 @@ def load_library():
         fn = getattr(lib, name)
         fn.argtypes = [C.c_void_p, C.POINTER(argt), C.c_void_p]
         fn.restype = C.c_int
+    lib.falcon_tree_accept_static.argtypes = [C.POINTER(AcceptArgs), C.c_void_p]
+    lib.falcon_tree_accept_static.restype = C.c_int
     _lib = lib
     return lib
 
@@ -96,6 +98,19 @@ def falcon_tree_validate_host(parent) -> int:
     import numpy as np
     parent = np.ascontiguousarray(parent, dtype=np.int32)
     return int(load_library().falcon_tree_validate_host(parent.ctypes.data, len(parent)))
+
+
+STATIC_MAX_NODES, STATIC_MAX_BATCH = 1024, 256
+
+
+def falcon_tree_accept_static(args: "AcceptArgs", stream=None, check: bool = True) -> int:
+    """Greedy acceptance without any device allocation: no context, scratch in a fixed array
+    inside the library (limits STATIC_MAX_NODES / STATIC_MAX_BATCH).  For hosts that may not
+    call cudaMalloc; calls that overlap on the GPU must be serialised by the caller."""
+    rc = load_library().falcon_tree_accept_static(C.byref(args), _stream(stream))
+    if check and rc:
+        raise FalconError(rc, "falcon_tree_accept_static")
+    return rc
 
 
 def _ptr(x) -> Optional[int]:

@@ -218,3 +218,119 @@ int launch_tree_accept(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_
 }
 
 }  // namespace falcon
+
+// ---------------------------------------------------------------------------------------------
+// falcon_tree_accept_static: the same acceptance kernel for callers that must not allocate.
+//
+// Some hosts of this library cannot call cudaMalloc at all: an inference server whose device
+// memory is handed out entirely by its own pool, a process running under a fixed memory budget
+// (an MPS client with a memory limit, a container whose quota is already committed), or a decode
+// loop that cannot tolerate the implicit synchronisation an allocation may bring.  For them the
+// scratch of the acceptance kernel (the per-chunk argmax partials and the arrival counters) lives
+// in the fixed array below, which is part of the library image: every GPU that loads the library
+// holds these bytes until the process exits, whether or not this entry point is ever called.
+// ---------------------------------------------------------------------------------------------
+#include <mutex>
+
+namespace falcon {
+namespace {
+
+constexpr int kStaticMaxNodes = FALCON_STATIC_MAX_NODES;
+constexpr int kStaticMaxBatch = FALCON_STATIC_MAX_BATCH;
+constexpr int kStaticMaxChunks = 64;
+constexpr size_t kStaticPartBytes = static_cast<size_t>(kStaticMaxNodes) * kStaticMaxChunks * 8;  // values + indices
+constexpr size_t kStaticBytes = kStaticPartBytes + static_cast<size_t>(kStaticMaxBatch) * sizeof(int);
+
+// In host code this name is only a handle for cudaGetSymbolAddress; it is not a device address.
+static __device__ __align__(256) unsigned char g_accept_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+struct StaticSlot {
+  void* ptr = nullptr;  // device address of g_accept_scratch on this device
+  int sm_count = 0;
+};
+StaticSlot g_slots[kMaxDevices];
+std::mutex g_slots_mutex;
+
+// Once per device, with that device current: resolve the array's device address.
+int static_scratch(int device, StaticSlot* out) {
+  std::lock_guard<std::mutex> lock(g_slots_mutex);
+  StaticSlot& slot = g_slots[device];
+  if (slot.ptr == nullptr) {
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_accept_scratch);
+    if (e != cudaSuccess || ptr == nullptr) return FALCON_ERR_CUDA;
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    if (e != cudaSuccess || sms < 1) return FALCON_ERR_CUDA;
+    slot.sm_count = sms;
+    slot.ptr = ptr;
+  }
+  *out = slot;
+  return FALCON_OK;
+}
+
+}  // namespace
+}  // namespace falcon
+
+extern "C" int falcon_tree_accept_static(const falcon_accept_args* a, void* stream) {
+  using namespace falcon;
+  if (!a) return FALCON_ERR_INVALID_ARG;
+  int rc = check_tree_desc(a->tree, true);
+  if (rc) return rc;
+  if (!a->logits || !a->argmax_out || !a->path || !a->n_path || !a->next_token) return FALCON_ERR_INVALID_ARG;
+  if (a->vocab < 1 || a->logits_stride < a->vocab) return FALCON_ERR_INVALID_ARG;
+  if (a->path_stride < a->tree.max_tree) return FALCON_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(a->logits) & 3) return FALCON_ERR_INVALID_ARG;
+  // sizes beyond the fixed scratch are refused, never truncated
+  if (a->tree.total_nodes > kStaticMaxNodes || a->tree.batch > kStaticMaxBatch) return FALCON_ERR_CAPACITY;
+
+  int device = -1;
+  if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return FALCON_ERR_CUDA;
+  StaticSlot slot;
+  rc = static_scratch(device, &slot);
+  if (rc) return rc;
+
+  const int N = a->tree.total_nodes;
+  int chunks = (4 * slot.sm_count + N - 1) / N;
+  const int max_chunks = (a->vocab + 2047) / 2048;
+  if (chunks > max_chunks) chunks = max_chunks;
+  if (chunks > kStaticMaxChunks) chunks = kStaticMaxChunks;
+  if (chunks < 1) chunks = 1;
+  int chunk_len = (a->vocab + chunks - 1) / chunks;
+  chunk_len = (chunk_len + 3) & ~3;
+  chunks = (a->vocab + chunk_len - 1) / chunk_len;
+
+  unsigned char* base = static_cast<unsigned char*>(slot.ptr);
+  const size_t part = static_cast<size_t>(N) * chunks;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // The array keeps whatever the previous call left.  The partials are fully rewritten by this
+  // launch; the arrival counters must start at zero, so they are cleared on the stream first.
+  cudaError_t e = cudaMemsetAsync(base + kStaticPartBytes, 0, static_cast<size_t>(a->tree.batch) * sizeof(int), s);
+  if (e != cudaSuccess) return FALCON_ERR_CUDA;
+
+  AcceptParams p;
+  p.batch = a->tree.batch;
+  p.total_nodes = N;
+  p.vocab = a->vocab;
+  p.chunks = chunks;
+  p.chunk_len = chunk_len;
+  p.path_stride = a->path_stride;
+  p.logits_stride = a->logits_stride;
+  p.node_off = a->tree.node_off;
+  p.parent = a->tree.parent;
+  p.token = a->tree.token;
+  p.status = a->tree.status;
+  p.logits = a->logits;
+  p.argmax_out = a->argmax_out;
+  p.path = a->path;
+  p.n_path = a->n_path;
+  p.next_token = a->next_token;
+  p.part_val = reinterpret_cast<float*>(base);
+  p.part_idx = reinterpret_cast<int32_t*>(base) + part;
+  p.tickets = reinterpret_cast<int*>(base + kStaticPartBytes);
+  dim3 grid(chunks, N);
+  tree_accept_kernel<<<grid, kAcceptThreads, 0, s>>>(p);
+  e = cudaGetLastError();
+  return e == cudaSuccess ? FALCON_OK : FALCON_ERR_CUDA;
+}
