@@ -1,7 +1,708 @@
-// placeholder until the tensor-core kernel lands
+// falcon_tree_attn, tensor-core kernel for sm_100a (head_dim 128, tree K/V in the cache).
+//
+// Work decomposition: one thread-block cluster per (sequence, KV head, tile of 128
+// query rows); query row m of a KV head is (tree node m / G, query head m % G), so
+// grouped-query heads share the K/V stream.  The cluster's CTAs split the key range
+// (prefix + tree) into contiguous runs of 64-key tiles; each CTA runs a flash-style
+// loop over its run and the cluster merges the partial (max, sum, O) through
+// distributed shared memory, so no partial ever goes to global memory.
+//
+// Inside a CTA (192 threads):
+//   warp 0    TMA producer: Q once, then K and V tiles (bf16, 128-byte swizzle) into a
+//             4-stage ring, completion on mbarriers.
+//   warp 1    one thread issues tcgen05.mma: S = Q.K^T (M=128, N=64, K=128) into one of
+//             two TMEM score buffers, and O += P.V (M=128, N=128, K=64) into the TMEM
+//             accumulator; tcgen05.commit signals the consumers.
+//   warps 2-5 one thread per query row: tcgen05.ld of the score row, tree mask from the
+//             node's ancestor bit set, online softmax with a lazily updated maximum (the
+//             accumulator is rescaled only when the row maximum grows by more than 2^8),
+//             P written as bf16 into swizzled shared memory for the second MMA.
+// Every mbarrier wait is bounded; a wait that runs out sets FALCON_DEV_TIMEOUT in the
+// status word, and the CTA still reaches the cluster barriers and frees its TMEM.
+#include <cuda.h>
+
+#include <mutex>
+#include <vector>
+
 #include "common.cuh"
+
 namespace falcon {
-bool tree_attn_tc_supports(const falcon_ctx*, const falcon_attn_args&) { return false; }
-int launch_tree_attn_tc(falcon_ctx*, const falcon_attn_args&, cudaStream_t) { return FALCON_ERR_UNSUPPORTED; }
-void tree_attn_tc_release(falcon_ctx*) {}
+namespace {
+
+constexpr int kD = 128;
+constexpr int kBM = 128;          // query rows per CTA (TMEM lanes)
+constexpr int kBN = 64;           // keys per tile
+constexpr int kStages = 4;
+constexpr int kTcThreads = 192;
+constexpr int kMaxSplits = 8;
+constexpr uint32_t kSpinLimit = 1u << 18;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units
+
+constexpr uint32_t kQBytes = kBM * kD * 2;         // 32 KB: two 64-column halves of 16 KB
+constexpr uint32_t kPBytes = kBM * kBN * 2;        // 16 KB per buffer
+constexpr uint32_t kTileBytes = kBN * kD * 2;      // 16 KB: two halves of 8 KB
+constexpr uint32_t kHalfTile = kBN * 128;          // 8 KB
+constexpr uint32_t kOffQ = 0;
+constexpr uint32_t kOffP = kOffQ + kQBytes;
+constexpr uint32_t kOffKV = kOffP + 2 * kPBytes;
+constexpr uint32_t kSmemBytes = kOffKV + kStages * 2 * kTileBytes;  // 196608
+constexpr uint32_t kSmemAlloc = kSmemBytes + 1024;                  // room to align the base to 1 KB
+constexpr uint32_t kTmemCols = 256;  // scores 2 x 64, accumulator 128
+constexpr uint32_t kTmemO = 128;
+
+// barrier indices
+enum {
+  kBarQ = 0,
+  kBarKFull = 1,                     // [kStages]
+  kBarVFull = kBarKFull + kStages,   // [kStages]
+  kBarKVEmpty = kBarVFull + kStages, // [kStages]
+  kBarSFull = kBarKVEmpty + kStages, // [2]
+  kBarSEmpty = kBarSFull + 2,        // [2]
+  kBarPFull = kBarSEmpty + 2,        // [2]
+  kBarPEmpty = kBarPFull + 2,        // [2]  also "P.V of tile j finished"
+  kBarODone = kBarPEmpty + 2,
+  kNumBars = kBarODone + 1
+};
+
+struct TcParams {
+  int32_t Hq, Hkv, G, s_cap, total_nodes;
+  float scale_log2;
+  const int32_t* node_off;
+  const int32_t* parent;
+  const int32_t* prefix_len;
+  int32_t* status;
+  const uint64_t* tree_mask;
+  __nv_bfloat16* out;
+};
+
+// ------------------------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("{ .reg .b64 t; mbarrier.arrive.shared::cta.b64 t, [%0]; }" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("{ .reg .b64 t; mbarrier.arrive.expect_tx.shared::cta.b64 t, [%0], %1; }" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+// Bounded wait: false when the limit ran out (or another thread already gave up).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if ((it & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+// Same, for a whole warp: every lane waits and the warp takes one decision.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  const bool ok = mbar_wait(bar, parity, abort_flag);
+  return __all_sync(0xffffffffu, ok);
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return static_cast<uint64_t>((addr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(lbo_bytes >> 4) << 16) |
+         (static_cast<uint64_t>(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// instruction descriptors: bf16 x bf16 -> fp32
+constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((kBN >> 3) << 17) | ((kBM >> 4) << 24);
+constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((kD >> 3) << 17) | ((kBM >> 4) << 24);
+
+#define FALCON_TMEM_LD32(taddr, r)                                                                                    \
+  asm volatile(                                                                                                       \
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19," \
+      "%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"                                                      \
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),   \
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),        \
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),       \
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])                     \
+      : "r"(taddr)                                                                                                    \
+      : "memory")
+
+#define FALCON_TMEM_ST32(taddr, r)                                                                                    \
+  asm volatile(                                                                                                       \
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,"  \
+      "%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};" ::"r"(r[0]),                                        \
+      "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),   \
+      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]),     \
+      "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]),     \
+      "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr)                                                                  \
+      : "memory")
+
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
+
+// 64 visibility bits for tree indices off .. off+63 of a 128-bit set; negative indices (prefix keys) are visible.
+__device__ __forceinline__ uint64_t window64(uint64_t lo, uint64_t hi, int off) {
+  if (off <= -64) return ~0ull;
+  if (off < 0) return ((1ull << (-off)) - 1ull) | (lo << (-off));
+  if (off == 0) return lo;
+  if (off < 64) return (lo >> off) | (hi << (64 - off));
+  if (off == 64) return hi;
+  if (off < 128) return hi >> (off - 64);
+  return 0ull;
+}
+
+// ------------------------------------------------------------------------------------ kernel
+__global__ void __launch_bounds__(kTcThreads, 1)
+tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                    const __grid_constant__ CUtensorMap tm_v, const TcParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) uint64_t s_bars[kNumBars];
+  __shared__ uint32_t s_tmem_base;
+  __shared__ float s_m[kBM], s_l[kBM];
+  __shared__ int s_abort;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_splits = gridDim.x, split = blockIdx.x;  // cluster = all CTAs of a row of the grid
+  const int kvh = blockIdx.y % p.Hkv, mtile = blockIdx.y / p.Hkv, b = blockIdx.z;
+  const int G = p.G;
+
+  const int node_base = p.node_off[b];
+  const int T_real = p.node_off[b + 1] - node_base;
+  const int T = min(T_real, FALCON_T_MAX);
+  const int rows_total = T * G;
+  if (mtile * kBM >= rows_total) return;  // same decision in every CTA of the cluster
+  const int n_valid = min(kBM, rows_total - mtile * kBM);
+  const int L = max(p.prefix_len[b], 0);
+  const int Lc = min(L, p.s_cap);
+  const int S_valid = min(L + T, p.s_cap);  // keys that exist below the cache capacity
+  const int n_tiles = (S_valid + kBN - 1) / kBN;
+  const int t_begin = (split * n_tiles) / n_splits;
+  const int t_end = ((split + 1) * n_tiles) / n_splits;
+  const int n_my = t_end - t_begin;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bars = smem_u32(s_bars);
+  auto bar = [&](int i) { return bars + 8u * static_cast<uint32_t>(i); };
+
+  if (tid == 0) {
+    s_abort = 0;
+    mbar_init(bar(kBarQ), 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bar(kBarKFull + s), 1);
+      mbar_init(bar(kBarVFull + s), 1);
+      mbar_init(bar(kBarKVEmpty + s), 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar(kBarSFull + s), 1);
+      mbar_init(bar(kBarSEmpty + s), 4);
+      mbar_init(bar(kBarPFull + s), 4);
+      mbar_init(bar(kBarPEmpty + s), 1);
+    }
+    mbar_init(bar(kBarODone), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (split == 0 && mtile == 0 && kvh == 0 && (L + T > p.s_cap || T_real > FALCON_T_MAX))
+      dev_status_or(p.status, b, FALCON_DEV_CAPACITY);
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = s_tmem_base;
+  volatile int* abort_flag = &s_abort;
+
+  if (warp == 0) {
+    // ================================ TMA producer ================================
+    if (lane == 0 && n_my > 0) {
+      const int node0 = node_base + mtile * (kBM / G);
+      mbar_expect_tx(bar(kBarQ), kQBytes);
+      tma_load_4d(smem_base + kOffQ, &tm_q, bar(kBarQ), 0, 0, kvh, node0);
+      tma_load_4d(smem_base + kOffQ + kQBytes / 2, &tm_q, bar(kBarQ), 64, 0, kvh, node0);
+      for (int j = 0; j < n_my; ++j) {
+        const int st = j % kStages, u = j / kStages;
+        if (u >= 1 && !mbar_wait(bar(kBarKVEmpty + st), (u - 1) & 1, abort_flag)) break;
+        const int k0 = (t_begin + j) * kBN;
+        const uint32_t kdst = smem_base + kOffKV + st * 2 * kTileBytes;
+        const uint32_t vdst = kdst + kTileBytes;
+        mbar_expect_tx(bar(kBarKFull + st), kTileBytes);
+        tma_load_4d(kdst, &tm_k, bar(kBarKFull + st), 0, k0, kvh, b);
+        tma_load_4d(kdst + kHalfTile, &tm_k, bar(kBarKFull + st), 64, k0, kvh, b);
+        mbar_expect_tx(bar(kBarVFull + st), kTileBytes);
+        tma_load_4d(vdst, &tm_v, bar(kBarVFull + st), 0, k0, kvh, b);
+        tma_load_4d(vdst + kHalfTile, &tm_v, bar(kBarVFull + st), 64, k0, kvh, b);
+      }
+    }
+  } else if (warp == 1) {
+    // ================================ MMA issuer ================================
+    if (lane == 0 && n_my > 0) {
+      bool ok = mbar_wait(bar(kBarQ), 0, abort_flag);
+      auto issue_pv = [&](int t) -> bool {
+        const int st = t % kStages, pb = t & 1;
+        if (!mbar_wait(bar(kBarPFull + pb), (t >> 1) & 1, abort_flag)) return false;
+        if (!mbar_wait(bar(kBarVFull + st), (t / kStages) & 1, abort_flag)) return false;
+        tc_fence_after();
+        const uint32_t pbase = smem_base + kOffP + pb * kPBytes;
+        const uint32_t vbase = smem_base + kOffKV + st * 2 * kTileBytes + kTileBytes;
+#pragma unroll
+        for (int kk = 0; kk < kBN / 16; ++kk) {
+          const uint64_t a = smem_desc(pbase + kk * 32, 16, 1024);            // P: K-major, 64 keys = one swizzle row
+          const uint64_t bd = smem_desc(vbase + kk * 2048, kHalfTile, 1024);  // V: MN-major, halves 8 KB apart
+          umma_bf16(tmem_base + kTmemO, a, bd, kIdescPV, (t > 0 || kk > 0) ? 1u : 0u);
+        }
+        umma_commit(bar(kBarKVEmpty + st));
+        umma_commit(bar(kBarPEmpty + pb));
+        return true;
+      };
+      for (int j = 0; ok && j < n_my; ++j) {
+        const int st = j % kStages, sb = j & 1;
+        if (!mbar_wait(bar(kBarKFull + st), (j / kStages) & 1, abort_flag)) { ok = false; break; }
+        if (j >= 2 && !mbar_wait(bar(kBarSEmpty + sb), ((j >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t qbase = smem_base + kOffQ;
+        const uint32_t kbase = smem_base + kOffKV + st * 2 * kTileBytes;
+#pragma unroll
+        for (int kk = 0; kk < kD / 16; ++kk) {
+          const uint64_t a = smem_desc(qbase + (kk >> 2) * (kQBytes / 2) + (kk & 3) * 32, 16, 1024);
+          const uint64_t bd = smem_desc(kbase + (kk >> 2) * kHalfTile + (kk & 3) * 32, 16, 1024);
+          umma_bf16(tmem_base + sb * kBN, a, bd, kIdescQK, kk > 0 ? 1u : 0u);
+        }
+        umma_commit(bar(kBarSFull + sb));
+        if (j >= 1 && !issue_pv(j - 1)) { ok = false; break; }
+      }
+      if (ok) ok = issue_pv(n_my - 1);
+      umma_commit(bar(kBarODone));  // fires once every MMA issued so far has finished
+    }
+  } else {
+    // ================================ softmax / correction ================================
+    const int q4 = warp & 3;
+    const int row = q4 * 32 + lane;
+    const bool valid = row < n_valid;
+    const bool warp_valid = q4 * 32 < n_valid;
+    const uint32_t tmem_lane = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16);
+    const int sm_tid = tid - 64;  // 0..127 over the four softmax warps
+
+    uint64_t anc_lo = 0, anc_hi = 0;
+    if (valid) {
+      const int node = (mtile * kBM + row) / G;
+      bool bad = false;
+      if (p.tree_mask) {
+        anc_lo = p.tree_mask[2 * static_cast<int64_t>(node_base + node)];
+        anc_hi = p.tree_mask[2 * static_cast<int64_t>(node_base + node) + 1];
+      } else {
+        bad = !ancestor_mask(p.parent + node_base, T, node, anc_lo, anc_hi);
+        if (node == 0 && p.parent[node_base] != -1) bad = true;
+      }
+      if (bad && split == 0 && kvh == 0) dev_status_or(p.status, b, FALCON_DEV_BAD_TREE);
+      const int nt = S_valid - Lc;  // tree keys that can be read (<= T)
+      if (nt < 64) {
+        anc_hi = 0;
+        anc_lo &= (nt <= 0) ? 0ull : ((1ull << nt) - 1ull);
+      } else if (nt < 128) {
+        anc_hi &= (nt == 64) ? 0ull : ((1ull << (nt - 64)) - 1ull);
+      }
+    }
+    float m_used = -INFINITY, l_sum = 0.f;
+
+    for (int j = 0; j < n_my; ++j) {
+      const int sb = j & 1, u2 = j >> 1, st = j % kStages;
+      const int k0 = (t_begin + j) * kBN;
+      if (!mbar_wait_warp(bar(kBarSFull + sb), u2 & 1, abort_flag)) break;
+      tc_fence_after();
+      uint32_t sr[64];
+      if (warp_valid) {
+        FALCON_TMEM_LD32(tmem_lane + sb * kBN, sr);
+        FALCON_TMEM_LD32(tmem_lane + sb * kBN + 32, (sr + 32));
+        tmem_wait_ld();
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(kBarSEmpty + sb));
+
+      // the sequence's last tile: rows of V past the last key may hold anything (0 x NaN = NaN in the MMA)
+      if (k0 + kBN > S_valid) {
+        if (!mbar_wait_warp(bar(kBarVFull + st), (j / kStages) & 1, abort_flag)) break;
+        const int nv = S_valid - k0;  // 1..63 rows are real
+        unsigned char* vtile = smem_raw + (smem_base - smem_u32(smem_raw)) + kOffKV + st * 2 * kTileBytes + kTileBytes;
+        const int chunks = (kBN - nv) * 8;
+        for (int c = sm_tid; c < 2 * chunks; c += 128) {
+          const int half = c / chunks, cc = c % chunks;
+          *reinterpret_cast<uint4*>(vtile + half * kHalfTile + nv * 128 + cc * 16) = make_uint4(0, 0, 0, 0);
+        }
+        fence_async_smem();
+      }
+
+      uint32_t pk[32];
+      float alpha = 1.f;
+      bool need_rescale = false;
+      if (valid) {
+        float s[64];
+        float tmax = -INFINITY;
+        if (k0 + kBN <= Lc) {
+#pragma unroll
+          for (int c = 0; c < 64; ++c) {
+            s[c] = __uint_as_float(sr[c]) * p.scale_log2;
+            tmax = fmaxf(tmax, s[c]);
+          }
+        } else {
+          const uint64_t vis = window64(anc_lo, anc_hi, k0 - Lc);
+#pragma unroll
+          for (int c = 0; c < 64; ++c) {
+            s[c] = ((vis >> c) & 1ull) ? __uint_as_float(sr[c]) * p.scale_log2 : -INFINITY;
+            tmax = fmaxf(tmax, s[c]);
+          }
+        }
+        if (m_used == -INFINITY) {
+          m_used = tmax;  // nothing accumulated yet for this row (O and l are zero)
+        } else if (tmax > m_used + kRescaleThreshold) {
+          alpha = ex2(m_used - tmax);
+          l_sum *= alpha;
+          m_used = tmax;
+          need_rescale = true;
+        }
+        const float m_eff = (m_used == -INFINITY) ? 0.f : m_used;
+        float add = 0.f;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const float p0 = ex2(s[2 * c] - m_eff), p1 = ex2(s[2 * c + 1] - m_eff);
+          add += p0 + p1;
+          const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+          pk[c] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        l_sum += add;
+      }
+
+      // P buffer free again?  (P.V of tile j-2 finished)
+      if (u2 >= 1 && !mbar_wait_warp(bar(kBarPEmpty + sb), (u2 - 1) & 1, abort_flag)) break;
+
+      // rare: the row maximum jumped; rescale the accumulator before this tile is added
+      if (warp_valid && __any_sync(0xffffffffu, need_rescale) && j > 0) {
+        if (!mbar_wait_warp(bar(kBarPEmpty + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag)) break;
+        tc_fence_after();
+#pragma unroll 1
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t o[32];
+          FALCON_TMEM_LD32(tmem_lane + kTmemO + ch * 32, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+          FALCON_TMEM_ST32(tmem_lane + kTmemO + ch * 32, o);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+      }
+
+      if (valid) {
+        const uint32_t prow = smem_base + kOffP + sb * kPBytes + row * 128;
+#pragma unroll
+        for (int c8 = 0; c8 < 8; ++c8) {
+          const uint32_t addr = prow + (static_cast<uint32_t>(c8 ^ (row & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[4 * c8]), "r"(pk[4 * c8 + 1]),
+                       "r"(pk[4 * c8 + 2]), "r"(pk[4 * c8 + 3])
+                       : "memory");
+        }
+      }
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(kBarPFull + sb));
+    }
+
+    // ---- this split's partial result into shared memory for the cluster merge ----
+    float* mb = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) + kOffKV);  // [col][row]
+    bool have = (n_my > 0) && !*abort_flag;
+    if (have) have = mbar_wait_warp(bar(kBarODone), 0, abort_flag);
+    tc_fence_after();
+    if (have && warp_valid) {
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t o[32];
+        FALCON_TMEM_LD32(tmem_lane + kTmemO + ch * 32, o);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) mb[(ch * 32 + c) * kBM + row] = __uint_as_float(o[c]);
+      }
+    }
+    s_m[row] = have ? m_used : -INFINITY;
+    s_l[row] = have ? l_sum : 0.f;
+  }
+
+  // ================================ cluster merge ================================
+  tc_fence_before();
+  __syncthreads();
+  if (s_abort && tid == 0) dev_status_or(p.status, b, FALCON_DEV_TIMEOUT);
+  cluster_sync_all();
+  {
+    const int rows_per = (n_valid + n_splits - 1) / n_splits;
+    const int row0 = split * rows_per;
+    const int rows_mine = max(0, min(n_valid, row0 + rows_per) - row0);
+    const uint32_t mb_local = smem_base + kOffKV;
+    const uint32_t m_local = smem_u32(s_m), l_local = smem_u32(s_l);
+    for (int item = tid; item < rows_mine * (kD / 8); item += kTcThreads) {
+      const int rl = item % rows_mine, cg = item / rows_mine;
+      const int row = row0 + rl;
+      float gm = -INFINITY;
+      for (int s = 0; s < n_splits; ++s) gm = fmaxf(gm, ld_cluster_f32(map_to_rank(m_local + 4 * row, s)));
+      float lsum = 0.f, acc[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) acc[c] = 0.f;
+      for (int s = 0; s < n_splits; ++s) {
+        const float ms = ld_cluster_f32(map_to_rank(m_local + 4 * row, s));
+        if (ms == -INFINITY) continue;
+        const float w = ex2(ms - gm);
+        lsum = fmaf(ld_cluster_f32(map_to_rank(l_local + 4 * row, s)), w, lsum);
+        const uint32_t src = map_to_rank(mb_local + 4u * static_cast<uint32_t>((cg * 8) * kBM + row), s);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) acc[c] = fmaf(ld_cluster_f32(src + 4u * c * kBM), w, acc[c]);
+      }
+      const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+      const int mg = mtile * kBM + row;
+      const int node = mg / G, head = kvh * G + mg % G;
+      __align__(16) __nv_bfloat162 pkd[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) pkd[c] = __floats2bfloat162_rn(acc[2 * c] * inv, acc[2 * c + 1] * inv);
+      *reinterpret_cast<uint4*>(p.out + (static_cast<int64_t>(node_base + node) * p.Hq + head) * kD + cg * 8) =
+          *reinterpret_cast<const uint4*>(pkd);
+    }
+  }
+  cluster_sync_all();  // nobody leaves while a peer may still read its shared memory
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------ host side
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn get_encode() {
+  static EncodeFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeFn>(ptr);
+  });
+  return fn;
+}
+
+struct TmapEntry {
+  const void* base;
+  uint64_t dims[4];
+  uint64_t strides[3];
+  uint32_t box[4];
+  CUtensorMap map;
+};
+
+struct TmapCache {
+  std::vector<TmapEntry> entries;
+};
+
+// 4-D bf16 tensor map with 128-byte swizzle; cached per (base, shape, strides, box).
+const CUtensorMap* get_tmap(falcon_ctx* ctx, const void* base, const uint64_t dims[4], const uint64_t strides[3],
+                            const uint32_t box[4]) {
+  if (!ctx->tmap_cache) ctx->tmap_cache = new TmapCache();
+  TmapCache* cache = static_cast<TmapCache*>(ctx->tmap_cache);
+  for (TmapEntry& e : cache->entries) {
+    if (e.base != base) continue;
+    bool same = true;
+    for (int i = 0; i < 4; ++i) same = same && e.dims[i] == dims[i] && e.box[i] == box[i];
+    for (int i = 0; i < 3; ++i) same = same && e.strides[i] == strides[i];
+    if (same) return &e.map;
+  }
+  EncodeFn enc = get_encode();
+  if (!enc) return nullptr;
+  if (cache->entries.size() >= 4096) cache->entries.clear();
+  TmapEntry e;
+  e.base = base;
+  for (int i = 0; i < 4; ++i) { e.dims[i] = dims[i]; e.box[i] = box[i]; }
+  for (int i = 0; i < 3; ++i) e.strides[i] = strides[i];
+  const cuuint32_t elem[4] = {1, 1, 1, 1};
+  alignas(64) CUtensorMap m;
+  CUresult r = enc(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, elem,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return nullptr;
+  e.map = m;
+  cache->entries.reserve(4096);  // pointers into the vector stay valid until it is cleared
+  cache->entries.push_back(e);
+  return &cache->entries.back().map;
+}
+
+bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+
+// Largest cluster size (number of KV splits) for which `units` clusters are co-resident.
+int pick_splits(falcon_ctx* ctx, int units, int max_tiles) {
+  static int resident[kMaxSplits + 1] = {0};
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  int best = 1;
+  for (int s = kMaxSplits; s >= 1; --s) {
+    if (s > max_tiles) continue;
+    if (resident[s] == 0) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(s, ctx->sm_count, 1);
+      cfg.blockDim = dim3(kTcThreads);
+      cfg.dynamicSmemBytes = kSmemAlloc;
+      cudaLaunchAttribute attr;
+      attr.id = cudaLaunchAttributeClusterDimension;
+      attr.val.clusterDim.x = s;
+      attr.val.clusterDim.y = 1;
+      attr.val.clusterDim.z = 1;
+      cfg.attrs = &attr;
+      cfg.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, tree_attn_tc_kernel, &cfg) != cudaSuccess) n = -1;
+      resident[s] = n > 0 ? n : -1;
+      cudaGetLastError();
+    }
+    if (resident[s] >= units) { best = s; break; }
+  }
+  return best;
+}
+
+}  // namespace
+
+bool tree_attn_tc_supports(const falcon_ctx* ctx, const falcon_attn_args& a) {
+  (void)ctx;
+  if (a.head_dim != kD) return false;
+  if (a.k_tree != nullptr) return false;
+  const int G = a.n_q_heads / a.n_kv_heads;
+  if (!is_pow2(G) || G > kBM) return false;
+  if (a.n_splits > kMaxSplits) return false;
+  if (a.tree.batch > 65535) return false;
+  return get_encode() != nullptr;
+}
+
+int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s) {
+  const int B = a.tree.batch, Hq = a.n_q_heads, Hkv = a.n_kv_heads, G = Hq / Hkv;
+  const int n_mtiles = (a.tree.max_tree * G + kBM - 1) / kBM;
+  if (static_cast<int64_t>(Hkv) * n_mtiles > 65535) return FALCON_ERR_CAPACITY;
+
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(kSmemAlloc));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaFuncSetAttribute(tree_attn_tc_kernel)");
+    attr_set = true;
+  }
+
+  // tensor maps: K/V cache [D, s_cap, Hkv, B], q [D, G, Hkv, N]
+  const uint64_t row_bytes = static_cast<uint64_t>(kD) * 2;
+  uint64_t kv_dims[4] = {static_cast<uint64_t>(kD), static_cast<uint64_t>(a.s_cap), static_cast<uint64_t>(Hkv),
+                         static_cast<uint64_t>(B)};
+  uint64_t kv_strides[3] = {static_cast<uint64_t>(a.kv_stride_s) * 2, static_cast<uint64_t>(a.kv_stride_h) * 2,
+                            static_cast<uint64_t>(a.kv_stride_b) * 2};
+  if (Hkv == 1 && kv_strides[1] == 0) kv_strides[1] = kv_strides[0] * a.s_cap;  // a size-1 dimension never strides
+  if (B == 1 && kv_strides[2] == 0) kv_strides[2] = kv_strides[1] * Hkv;
+  const uint32_t kv_box[4] = {64, static_cast<uint32_t>(kBN), 1, 1};
+  uint64_t q_dims[4] = {static_cast<uint64_t>(kD), static_cast<uint64_t>(G), static_cast<uint64_t>(Hkv),
+                        static_cast<uint64_t>(a.tree.total_nodes)};
+  uint64_t q_strides[3] = {row_bytes, row_bytes * G, row_bytes * Hq};
+  const uint32_t q_box[4] = {64, static_cast<uint32_t>(G), 1, static_cast<uint32_t>(kBM / G)};
+  const CUtensorMap* tq = get_tmap(ctx, a.q, q_dims, q_strides, q_box);
+  const CUtensorMap* tk = get_tmap(ctx, a.k_cache, kv_dims, kv_strides, kv_box);
+  const CUtensorMap* tv = get_tmap(ctx, a.v_cache, kv_dims, kv_strides, kv_box);
+  if (!tq || !tk || !tv) {
+    ctx->last_error = "cuTensorMapEncodeTiled failed";
+    return FALCON_ERR_CUDA;
+  }
+  const CUtensorMap mq = *tq, mk = *tk, mv = *tv;  // copies: later cache growth must not move what we pass
+
+  const int max_tiles = (a.tree.max_prefix_len + a.tree.max_tree + kBN - 1) / kBN;
+  int splits = a.n_splits;
+  if (splits == 0) splits = pick_splits(ctx, Hkv * n_mtiles * B, max_tiles > 0 ? max_tiles : 1);
+  if (splits < 1) splits = 1;
+
+  TcParams p;
+  p.Hq = Hq;
+  p.Hkv = Hkv;
+  p.G = G;
+  p.s_cap = a.s_cap;
+  p.total_nodes = a.tree.total_nodes;
+  p.scale_log2 = a.sm_scale * kLog2e;
+  p.node_off = a.tree.node_off;
+  p.parent = a.tree.parent;
+  p.prefix_len = a.tree.prefix_len;
+  p.status = a.tree.status;
+  p.tree_mask = a.tree_mask;
+  p.out = static_cast<__nv_bfloat16*>(a.out);
+
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(splits, Hkv * n_mtiles, B);
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = kSmemAlloc;
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = splits;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, mq, mk, mv, p);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "tree_attn_tc_kernel launch");
+  return FALCON_OK;
+}
+
+void tree_attn_tc_release(falcon_ctx* ctx) {
+  if (ctx->tmap_cache) {
+    delete static_cast<TmapCache*>(ctx->tmap_cache);
+    ctx->tmap_cache = nullptr;
+  }
+}
+
 }  // namespace falcon
