@@ -4,21 +4,25 @@
 // query rows); query row m of a KV head is (tree node m / G, query head m % G), so
 // grouped-query heads share the K/V stream.  The cluster's CTAs split the key range
 // (prefix + tree) into contiguous runs of 64-key tiles; each CTA runs a flash-style
-// loop over its run and the cluster merges the partial (max, sum, O) through
-// distributed shared memory, so no partial ever goes to global memory.
+// loop over its run, then pushes its partial (max, sum, O) rows into the shared
+// memory of the CTA that owns them (distributed shared memory), one cluster barrier,
+// and every CTA normalises and stores its share of the rows.  No partial result
+// touches global memory.
 //
 // Inside a CTA (192 threads):
-//   warp 0    TMA producer: Q once, then K and V tiles (bf16, 128-byte swizzle) into a
-//             4-stage ring, completion on mbarriers.
-//   warp 1    one thread issues tcgen05.mma: S = Q.K^T (M=128, N=64, K=128) into one of
-//             two TMEM score buffers, and O += P.V (M=128, N=128, K=64) into the TMEM
-//             accumulator; tcgen05.commit signals the consumers.
-//   warps 2-5 one thread per query row: tcgen05.ld of the score row, tree mask from the
-//             node's ancestor bit set, online softmax with a lazily updated maximum (the
-//             accumulator is rescaled only when the row maximum grows by more than 2^8),
-//             P written as bf16 into swizzled shared memory for the second MMA.
+//   warp 0    TMA producer: K and V tiles (bf16, 128-byte swizzle) into a 4-stage ring,
+//             completion on mbarriers; the first loads are issued before anything else.
+//   warp 1    one thread issues tcgen05.mma.  Both A operands live in tensor memory:
+//             S = Q.K^T (M=128, N=64, K=128) reads Q from TMEM and the K tile from shared
+//             memory; O += P.V (M=128, N=128, K=64) reads P from TMEM and the V tile from
+//             shared memory.  tcgen05.commit signals the consumers.
+//   warps 2-5 one thread per query row: loads its q row from global memory into TMEM once;
+//             per tile tcgen05.ld of the score row, tree mask from the node's ancestor bit
+//             set, online softmax with a lazily updated maximum (the accumulator is
+//             rescaled only when the row maximum grows by more than 2^8), P written back
+//             to TMEM as packed bf16.
 // Every mbarrier wait is bounded; a wait that runs out sets FALCON_DEV_TIMEOUT in the
-// status word, and the CTA still reaches the cluster barriers and frees its TMEM.
+// status word, and the CTA still reaches the cluster barrier and frees its TMEM.
 #include <cuda.h>
 
 #include <mutex>
@@ -38,21 +42,28 @@ constexpr int kMaxSplits = 8;
 constexpr uint32_t kSpinLimit = 1u << 18;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
-constexpr uint32_t kQBytes = kBM * kD * 2;         // 32 KB: two 64-column halves of 16 KB
-constexpr uint32_t kPBytes = kBM * kBN * 2;        // 16 KB per buffer
-constexpr uint32_t kTileBytes = kBN * kD * 2;      // 16 KB: two halves of 8 KB
+constexpr uint32_t kTileBytes = kBN * kD * 2;      // 16 KB: two 64-column halves of 8 KB
 constexpr uint32_t kHalfTile = kBN * 128;          // 8 KB
-constexpr uint32_t kOffQ = 0;
-constexpr uint32_t kOffP = kOffQ + kQBytes;
-constexpr uint32_t kOffKV = kOffP + 2 * kPBytes;
-constexpr uint32_t kSmemBytes = kOffKV + kStages * 2 * kTileBytes;  // 196608
-constexpr uint32_t kSmemAlloc = kSmemBytes + 1024;                  // room to align the base to 1 KB
-constexpr uint32_t kTmemCols = 256;  // scores 2 x 64, accumulator 128
-constexpr uint32_t kTmemO = 128;
+constexpr uint32_t kOffKV = 0;
+constexpr uint32_t kKVBytes = kStages * 2 * kTileBytes;  // 128 KB
+// merge buffer: partial rows pushed by the cluster's CTAs, [split][row_local] rows of kMrgPitch floats
+constexpr int kMrgRows = kBM + kMaxSplits;          // rows_per * n_splits <= n_valid + n_splits - 1
+constexpr int kMrgPitch = kD + 4;                   // 528-byte rows: 16-byte stores of 32 lanes spread over all banks
+constexpr uint32_t kOffMrg = kOffKV + kKVBytes;
+constexpr uint32_t kMrgBytes = kMrgRows * kMrgPitch * 4;
+constexpr uint32_t kOffML = kOffMrg + kMrgBytes;    // float2 (max, sum) per merge row
+constexpr uint32_t kSmemBytes = kOffML + kMrgRows * 8;
+constexpr uint32_t kSmemAlloc = kSmemBytes + 1024;  // room to align the base to 1 KB
 
-// barrier indices
+// tensor memory columns (32-bit each, 128 lanes)
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kTmemO = 0;      // 128 columns: fp32 accumulator
+constexpr uint32_t kTmemS = 128;    // 2 x 64 columns: fp32 scores
+constexpr uint32_t kTmemP = 256;    // 2 x 32 columns: bf16 pairs
+constexpr uint32_t kTmemQ = 320;    // 64 columns: bf16 pairs
+
 enum {
-  kBarQ = 0,
+  kBarQ = 0,                         // q rows are in TMEM (4 warps)
   kBarKFull = 1,                     // [kStages]
   kBarVFull = kBarKFull + kStages,   // [kStages]
   kBarKVEmpty = kBarVFull + kStages, // [kStages]
@@ -72,6 +83,7 @@ struct TcParams {
   const int32_t* prefix_len;
   int32_t* status;
   const uint64_t* tree_mask;
+  const __nv_bfloat16* q;
   __nv_bfloat16* out;
 };
 
@@ -103,7 +115,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   *abort_flag = 1;
   return false;
 }
-
 // Same, for a whole warp: every lane waits and the warp takes one decision.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   const bool ok = mbar_wait(bar, parity, abort_flag);
@@ -117,6 +128,9 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
 }
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -125,11 +139,12 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
+// D[tmem] (+)= A[tmem] . B[smem]
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
   asm volatile(
-      "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p; }" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 
@@ -139,7 +154,7 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
          (static_cast<uint64_t>(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
-// instruction descriptors: bf16 x bf16 -> fp32
+// instruction descriptors: bf16 x bf16 -> fp32, A K-major; B K-major (K tile) or MN-major (V tile)
 constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((kBN >> 3) << 17) | ((kBM >> 4) << 24);
 constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((kD >> 3) << 17) | ((kBM >> 4) << 24);
 
@@ -182,10 +197,12 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t ra
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
   return r;
 }
-__device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
-  return v;
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float a, float b, float c, float d) {
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
+               : "memory");
+}
+__device__ __forceinline__ void st_cluster_v2(uint32_t addr, float a, float b) {
+  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
 }
 
 // 64 visibility bits for tree indices off .. off+63 of a 128-bit set; negative indices (prefix keys) are visible.
@@ -201,12 +218,11 @@ __device__ __forceinline__ uint64_t window64(uint64_t lo, uint64_t hi, int off) 
 
 // ------------------------------------------------------------------------------------ kernel
 __global__ void __launch_bounds__(kTcThreads, 1)
-tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                    const __grid_constant__ CUtensorMap tm_v, const TcParams p) {
+tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                    const TcParams p) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t s_bars[kNumBars];
   __shared__ uint32_t s_tmem_base;
-  __shared__ float s_m[kBM], s_l[kBM];
   __shared__ int s_abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -214,13 +230,18 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int kvh = blockIdx.y % p.Hkv, mtile = blockIdx.y / p.Hkv, b = blockIdx.z;
   const int G = p.G;
 
+  if (tid == 0) {
+    prefetch_tmap(&tm_k);
+    prefetch_tmap(&tm_v);
+  }
   const int node_base = p.node_off[b];
   const int T_real = p.node_off[b + 1] - node_base;
+  const int L_raw = p.prefix_len[b];
   const int T = min(T_real, FALCON_T_MAX);
   const int rows_total = T * G;
   if (mtile * kBM >= rows_total) return;  // same decision in every CTA of the cluster
   const int n_valid = min(kBM, rows_total - mtile * kBM);
-  const int L = max(p.prefix_len[b], 0);
+  const int L = max(L_raw, 0);
   const int Lc = min(L, p.s_cap);
   const int S_valid = min(L + T, p.s_cap);  // keys that exist below the cache capacity
   const int n_tiles = (S_valid + kBN - 1) / kBN;
@@ -229,50 +250,84 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int n_my = t_end - t_begin;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   const uint32_t bars = smem_u32(s_bars);
   auto bar = [&](int i) { return bars + 8u * static_cast<uint32_t>(i); };
+  volatile int* abort_flag = &s_abort;
 
-  if (tid == 0) {
-    s_abort = 0;
-    mbar_init(bar(kBarQ), 1);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(bar(kBarKFull + s), 1);
-      mbar_init(bar(kBarVFull + s), 1);
-      mbar_init(bar(kBarKVEmpty + s), 1);
-    }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(bar(kBarSFull + s), 1);
-      mbar_init(bar(kBarSEmpty + s), 4);
-      mbar_init(bar(kBarPFull + s), 4);
-      mbar_init(bar(kBarPEmpty + s), 1);
-    }
-    mbar_init(bar(kBarODone), 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    if (split == 0 && mtile == 0 && kvh == 0 && (L + T > p.s_cap || T_real > FALCON_T_MAX))
-      dev_status_or(p.status, b, FALCON_DEV_CAPACITY);
-  }
+  // merge geometry: CTA `rank` owns rows [rank * rows_per, ...) of the tile
+  const int rows_per = (n_valid + n_splits - 1) / n_splits;
+
   if (warp == 0) {
+    if (lane == 0) {
+      s_abort = 0;
+      mbar_init(bar(kBarQ), 4);
+      for (int s = 0; s < kStages; ++s) {
+        mbar_init(bar(kBarKFull + s), 1);
+        mbar_init(bar(kBarVFull + s), 1);
+        mbar_init(bar(kBarKVEmpty + s), 1);
+      }
+      for (int s = 0; s < 2; ++s) {
+        mbar_init(bar(kBarSFull + s), 1);
+        mbar_init(bar(kBarSEmpty + s), 4);
+        mbar_init(bar(kBarPFull + s), 4);
+        mbar_init(bar(kBarPEmpty + s), 1);
+      }
+      mbar_init(bar(kBarODone), 1);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      // first ring fill right away: these loads need nothing but the barriers this thread just made
+      const int pre = min(n_my, kStages);
+      for (int j = 0; j < pre; ++j) {
+        const int k0 = (t_begin + j) * kBN;
+        const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
+        const uint32_t vdst = kdst + kTileBytes;
+        mbar_expect_tx(bar(kBarKFull + j), kTileBytes);
+        tma_load_4d(kdst, &tm_k, bar(kBarKFull + j), 0, k0, kvh, b);
+        tma_load_4d(kdst + kHalfTile, &tm_k, bar(kBarKFull + j), 64, k0, kvh, b);
+        mbar_expect_tx(bar(kBarVFull + j), kTileBytes);
+        tma_load_4d(vdst, &tm_v, bar(kBarVFull + j), 0, k0, kvh, b);
+        tma_load_4d(vdst + kHalfTile, &tm_v, bar(kBarVFull + j), 64, k0, kvh, b);
+      }
+      if (split == 0 && mtile == 0 && kvh == 0 && (L + T > p.s_cap || T_real > FALCON_T_MAX))
+        dev_status_or(p.status, b, FALCON_DEV_CAPACITY);
+    }
+    __syncwarp();
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
                  "r"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+
+  // softmax threads fetch their q row while the rest sets up
+  const int q4 = warp & 3;
+  const int row = q4 * 32 + lane;
+  const bool is_sm = warp >= 2;
+  const bool valid = is_sm && row < n_valid;
+  const bool warp_valid = is_sm && q4 * 32 < n_valid;
+  uint4 qreg[16];
+  if (warp_valid) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) qreg[i] = make_uint4(0, 0, 0, 0);
+    if (valid) {
+      const int mg = mtile * kBM + row;
+      const uint4* src = reinterpret_cast<const uint4*>(
+          p.q + (static_cast<int64_t>(node_base + mg / G) * p.Hq + kvh * G + mg % G) * kD);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) qreg[i] = __ldg(src + i);
+    }
+  }
+
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = s_tmem_base;
-  volatile int* abort_flag = &s_abort;
 
   if (warp == 0) {
-    // ================================ TMA producer ================================
-    if (lane == 0 && n_my > 0) {
-      const int node0 = node_base + mtile * (kBM / G);
-      mbar_expect_tx(bar(kBarQ), kQBytes);
-      tma_load_4d(smem_base + kOffQ, &tm_q, bar(kBarQ), 0, 0, kvh, node0);
-      tma_load_4d(smem_base + kOffQ + kQBytes / 2, &tm_q, bar(kBarQ), 64, 0, kvh, node0);
-      for (int j = 0; j < n_my; ++j) {
+    // ================================ TMA producer (ring refills) ================================
+    if (lane == 0) {
+      for (int j = kStages; j < n_my; ++j) {
         const int st = j % kStages, u = j / kStages;
-        if (u >= 1 && !mbar_wait(bar(kBarKVEmpty + st), (u - 1) & 1, abort_flag)) break;
+        if (!mbar_wait(bar(kBarKVEmpty + st), (u - 1) & 1, abort_flag)) break;
         const int k0 = (t_begin + j) * kBN;
         const uint32_t kdst = smem_base + kOffKV + st * 2 * kTileBytes;
         const uint32_t vdst = kdst + kTileBytes;
@@ -290,16 +345,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       bool ok = mbar_wait(bar(kBarQ), 0, abort_flag);
       auto issue_pv = [&](int t) -> bool {
         const int st = t % kStages, pb = t & 1;
-        if (!mbar_wait(bar(kBarPFull + pb), (t >> 1) & 1, abort_flag)) return false;
         if (!mbar_wait(bar(kBarVFull + st), (t / kStages) & 1, abort_flag)) return false;
+        if (!mbar_wait(bar(kBarPFull + pb), (t >> 1) & 1, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t pbase = smem_base + kOffP + pb * kPBytes;
         const uint32_t vbase = smem_base + kOffKV + st * 2 * kTileBytes + kTileBytes;
 #pragma unroll
         for (int kk = 0; kk < kBN / 16; ++kk) {
-          const uint64_t a = smem_desc(pbase + kk * 32, 16, 1024);            // P: K-major, 64 keys = one swizzle row
-          const uint64_t bd = smem_desc(vbase + kk * 2048, kHalfTile, 1024);  // V: MN-major, halves 8 KB apart
-          umma_bf16(tmem_base + kTmemO, a, bd, kIdescPV, (t > 0 || kk > 0) ? 1u : 0u);
+          // P: 16 keys = 8 packed columns; V: MN-major, 16 keys = 2 KB, the two 64-column halves 8 KB apart
+          const uint64_t bd = smem_desc(vbase + kk * 2048, kHalfTile, 1024);
+          umma_bf16_ts(tmem_base + kTmemO, tmem_base + kTmemP + pb * 32 + kk * 8, bd, kIdescPV,
+                       (t > 0 || kk > 0) ? 1u : 0u);
         }
         umma_commit(bar(kBarKVEmpty + st));
         umma_commit(bar(kBarPEmpty + pb));
@@ -310,13 +365,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (!mbar_wait(bar(kBarKFull + st), (j / kStages) & 1, abort_flag)) { ok = false; break; }
         if (j >= 2 && !mbar_wait(bar(kBarSEmpty + sb), ((j >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t qbase = smem_base + kOffQ;
         const uint32_t kbase = smem_base + kOffKV + st * 2 * kTileBytes;
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
-          const uint64_t a = smem_desc(qbase + (kk >> 2) * (kQBytes / 2) + (kk & 3) * 32, 16, 1024);
+          // K tile: K-major, 16 head-dim columns = 32 bytes inside the 128-byte swizzle row
           const uint64_t bd = smem_desc(kbase + (kk >> 2) * kHalfTile + (kk & 3) * 32, 16, 1024);
-          umma_bf16(tmem_base + sb * kBN, a, bd, kIdescQK, kk > 0 ? 1u : 0u);
+          umma_bf16_ts(tmem_base + kTmemS + sb * kBN, tmem_base + kTmemQ + kk * 8, bd, kIdescQK, kk > 0 ? 1u : 0u);
         }
         umma_commit(bar(kBarSFull + sb));
         if (j >= 1 && !issue_pv(j - 1)) { ok = false; break; }
@@ -326,12 +380,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
   } else {
     // ================================ softmax / correction ================================
-    const int q4 = warp & 3;
-    const int row = q4 * 32 + lane;
-    const bool valid = row < n_valid;
-    const bool warp_valid = q4 * 32 < n_valid;
     const uint32_t tmem_lane = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16);
     const int sm_tid = tid - 64;  // 0..127 over the four softmax warps
+
+    // q row -> TMEM (bf16 pairs, 64 columns)
+    if (warp_valid) {
+      const uint32_t* qw = reinterpret_cast<const uint32_t*>(qreg);
+      FALCON_TMEM_ST32(tmem_lane + kTmemQ, qw);
+      FALCON_TMEM_ST32(tmem_lane + kTmemQ + 32, (qw + 32));
+      tmem_wait_st();
+    }
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar(kBarQ));
 
     uint64_t anc_lo = 0, anc_hi = 0;
     if (valid) {
@@ -354,6 +415,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
     }
     float m_used = -INFINITY, l_sum = 0.f;
+    const float scale = p.scale_log2;
 
     for (int j = 0; j < n_my; ++j) {
       const int sb = j & 1, u2 = j >> 1, st = j % kStages;
@@ -362,8 +424,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       tc_fence_after();
       uint32_t sr[64];
       if (warp_valid) {
-        FALCON_TMEM_LD32(tmem_lane + sb * kBN, sr);
-        FALCON_TMEM_LD32(tmem_lane + sb * kBN + 32, (sr + 32));
+        FALCON_TMEM_LD32(tmem_lane + kTmemS + sb * kBN, sr);
+        FALCON_TMEM_LD32(tmem_lane + kTmemS + sb * kBN + 32, (sr + 32));
         tmem_wait_ld();
       }
       tc_fence_before();
@@ -374,7 +436,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (k0 + kBN > S_valid) {
         if (!mbar_wait_warp(bar(kBarVFull + st), (j / kStages) & 1, abort_flag)) break;
         const int nv = S_valid - k0;  // 1..63 rows are real
-        unsigned char* vtile = smem_raw + (smem_base - smem_u32(smem_raw)) + kOffKV + st * 2 * kTileBytes + kTileBytes;
+        unsigned char* vtile = smem_gen + kOffKV + st * 2 * kTileBytes + kTileBytes;
         const int chunks = (kBN - nv) * 8;
         for (int c = sm_tid; c < 2 * chunks; c += 128) {
           const int half = c / chunks, cc = c % chunks;
@@ -392,14 +454,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (k0 + kBN <= Lc) {
 #pragma unroll
           for (int c = 0; c < 64; ++c) {
-            s[c] = __uint_as_float(sr[c]) * p.scale_log2;
+            s[c] = __uint_as_float(sr[c]) * scale;
             tmax = fmaxf(tmax, s[c]);
           }
         } else {
           const uint64_t vis = window64(anc_lo, anc_hi, k0 - Lc);
 #pragma unroll
           for (int c = 0; c < 64; ++c) {
-            s[c] = ((vis >> c) & 1ull) ? __uint_as_float(sr[c]) * p.scale_log2 : -INFINITY;
+            s[c] = ((vis >> c) & 1ull) ? __uint_as_float(sr[c]) * scale : -INFINITY;
             tmax = fmaxf(tmax, s[c]);
           }
         }
@@ -412,15 +474,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           need_rescale = true;
         }
         const float m_eff = (m_used == -INFINITY) ? 0.f : m_used;
-        float add = 0.f;
+        float add0 = 0.f, add1 = 0.f;
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
           const float p0 = ex2(s[2 * c] - m_eff), p1 = ex2(s[2 * c + 1] - m_eff);
-          add += p0 + p1;
+          add0 += p0;
+          add1 += p1;
           const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
           pk[c] = *reinterpret_cast<const uint32_t*>(&h);
         }
-        l_sum += add;
+        l_sum += add0 + add1;
+      } else {
+#pragma unroll
+        for (int c = 0; c < 32; ++c) pk[c] = 0u;
       }
 
       // P buffer free again?  (P.V of tile j-2 finished)
@@ -439,83 +505,104 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
           FALCON_TMEM_ST32(tmem_lane + kTmemO + ch * 32, o);
         }
-        tmem_wait_st();
-        tc_fence_before();
       }
 
-      if (valid) {
-        const uint32_t prow = smem_base + kOffP + sb * kPBytes + row * 128;
-#pragma unroll
-        for (int c8 = 0; c8 < 8; ++c8) {
-          const uint32_t addr = prow + (static_cast<uint32_t>(c8 ^ (row & 7)) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[4 * c8]), "r"(pk[4 * c8 + 1]),
-                       "r"(pk[4 * c8 + 2]), "r"(pk[4 * c8 + 3])
-                       : "memory");
-        }
+      if (warp_valid) {
+        FALCON_TMEM_ST32(tmem_lane + kTmemP + sb * 32, pk);
+        tmem_wait_st();
       }
-      fence_async_smem();
+      tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(kBarPFull + sb));
     }
 
-    // ---- this split's partial result into shared memory for the cluster merge ----
-    float* mb = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) + kOffKV);  // [col][row]
+    // ---- this split's partial rows: straight to global (one split) or pushed to their owner ----
     bool have = (n_my > 0) && !*abort_flag;
     if (have) have = mbar_wait_warp(bar(kBarODone), 0, abort_flag);
     tc_fence_after();
-    if (have && warp_valid) {
+    if (warp_valid) {
+      const bool write = have && valid;
+      if (n_splits == 1) {
+        const float inv = (write && l_sum > 0.f) ? 1.f / l_sum : 0.f;
+        const int mg = mtile * kBM + row;
+        __nv_bfloat16* dst = p.out + (static_cast<int64_t>(node_base + mg / G) * p.Hq + kvh * G + mg % G) * kD;
 #pragma unroll 1
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t o[32];
-        FALCON_TMEM_LD32(tmem_lane + kTmemO + ch * 32, o);
-        tmem_wait_ld();
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t o[32];
+          FALCON_TMEM_LD32(tmem_lane + kTmemO + ch * 32, o);
+          tmem_wait_ld();
+          if (valid) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) mb[(ch * 32 + c) * kBM + row] = __uint_as_float(o[c]);
+            for (int c8 = 0; c8 < 4; ++c8) {
+              __align__(16) __nv_bfloat162 h[4];
+#pragma unroll
+              for (int c = 0; c < 4; ++c)
+                h[c] = __floats2bfloat162_rn(__uint_as_float(o[8 * c8 + 2 * c]) * inv,
+                                             __uint_as_float(o[8 * c8 + 2 * c + 1]) * inv);
+              *reinterpret_cast<uint4*>(dst + ch * 32 + c8 * 8) = *reinterpret_cast<const uint4*>(h);
+            }
+          }
+        }
+      } else {
+        const int owner = valid ? row / rows_per : 0;
+        const int slot = split * rows_per + (valid ? row % rows_per : 0);
+        const uint32_t dst = map_to_rank(smem_base + kOffMrg + static_cast<uint32_t>(slot) * (kMrgPitch * 4), owner);
+        if (valid)
+          st_cluster_v2(map_to_rank(smem_base + kOffML + static_cast<uint32_t>(slot) * 8, owner),
+                        write ? m_used : -INFINITY, write ? l_sum : 0.f);
+        if (have) {
+#pragma unroll 1
+          for (int ch = 0; ch < 4; ++ch) {
+            uint32_t o[32];
+            FALCON_TMEM_LD32(tmem_lane + kTmemO + ch * 32, o);
+            tmem_wait_ld();
+            if (valid) {
+#pragma unroll
+              for (int c4 = 0; c4 < 8; ++c4)
+                st_cluster_v4(dst + (ch * 32 + c4 * 4) * 4, __uint_as_float(o[4 * c4]), __uint_as_float(o[4 * c4 + 1]),
+                              __uint_as_float(o[4 * c4 + 2]), __uint_as_float(o[4 * c4 + 3]));
+            }
+          }
+        }
       }
     }
-    s_m[row] = have ? m_used : -INFINITY;
-    s_l[row] = have ? l_sum : 0.f;
   }
 
   // ================================ cluster merge ================================
   tc_fence_before();
   __syncthreads();
   if (s_abort && tid == 0) dev_status_or(p.status, b, FALCON_DEV_TIMEOUT);
-  cluster_sync_all();
-  {
-    const int rows_per = (n_valid + n_splits - 1) / n_splits;
+  if (n_splits > 1) {
+    cluster_sync_all();  // every CTA's rows have landed in their owner's shared memory
     const int row0 = split * rows_per;
     const int rows_mine = max(0, min(n_valid, row0 + rows_per) - row0);
-    const uint32_t mb_local = smem_base + kOffKV;
-    const uint32_t m_local = smem_u32(s_m), l_local = smem_u32(s_l);
-    for (int item = tid; item < rows_mine * (kD / 8); item += kTcThreads) {
-      const int rl = item % rows_mine, cg = item / rows_mine;
-      const int row = row0 + rl;
+    const float* mrg = reinterpret_cast<const float*>(smem_gen + kOffMrg);
+    const float2* ml = reinterpret_cast<const float2*>(smem_gen + kOffML);
+    for (int item = tid; item < rows_mine * (kD / 4); item += kTcThreads) {
+      const int rl = item / (kD / 4), c4 = item % (kD / 4);
       float gm = -INFINITY;
-      for (int s = 0; s < n_splits; ++s) gm = fmaxf(gm, ld_cluster_f32(map_to_rank(m_local + 4 * row, s)));
-      float lsum = 0.f, acc[8];
-#pragma unroll
-      for (int c = 0; c < 8; ++c) acc[c] = 0.f;
+      for (int s = 0; s < n_splits; ++s) gm = fmaxf(gm, ml[s * rows_per + rl].x);
+      float lsum = 0.f, a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
       for (int s = 0; s < n_splits; ++s) {
-        const float ms = ld_cluster_f32(map_to_rank(m_local + 4 * row, s));
-        if (ms == -INFINITY) continue;
-        const float w = ex2(ms - gm);
-        lsum = fmaf(ld_cluster_f32(map_to_rank(l_local + 4 * row, s)), w, lsum);
-        const uint32_t src = map_to_rank(mb_local + 4u * static_cast<uint32_t>((cg * 8) * kBM + row), s);
-#pragma unroll
-        for (int c = 0; c < 8; ++c) acc[c] = fmaf(ld_cluster_f32(src + 4u * c * kBM), w, acc[c]);
+        const float2 m_l = ml[s * rows_per + rl];
+        if (m_l.x == -INFINITY) continue;
+        const float w = ex2(m_l.x - gm);
+        lsum = fmaf(m_l.y, w, lsum);
+        const float4 x = *reinterpret_cast<const float4*>(mrg + (s * rows_per + rl) * kMrgPitch + c4 * 4);
+        a0 = fmaf(x.x, w, a0);
+        a1 = fmaf(x.y, w, a1);
+        a2 = fmaf(x.z, w, a2);
+        a3 = fmaf(x.w, w, a3);
       }
       const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-      const int mg = mtile * kBM + row;
-      const int node = mg / G, head = kvh * G + mg % G;
-      __align__(16) __nv_bfloat162 pkd[4];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) pkd[c] = __floats2bfloat162_rn(acc[2 * c] * inv, acc[2 * c + 1] * inv);
-      *reinterpret_cast<uint4*>(p.out + (static_cast<int64_t>(node_base + node) * p.Hq + head) * kD + cg * 8) =
-          *reinterpret_cast<const uint4*>(pkd);
+      const int mg = mtile * kBM + row0 + rl;
+      __align__(8) __nv_bfloat162 h[2];
+      h[0] = __floats2bfloat162_rn(a0 * inv, a1 * inv);
+      h[1] = __floats2bfloat162_rn(a2 * inv, a3 * inv);
+      *reinterpret_cast<uint2*>(p.out + (static_cast<int64_t>(node_base + mg / G) * p.Hq + kvh * G + mg % G) * kD +
+                                c4 * 4) = *reinterpret_cast<const uint2*>(h);
     }
   }
-  cluster_sync_all();  // nobody leaves while a peer may still read its shared memory
   if (warp == 0) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
@@ -640,8 +727,7 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
     attr_set = true;
   }
 
-  // tensor maps: K/V cache [D, s_cap, Hkv, B], q [D, G, Hkv, N]
-  const uint64_t row_bytes = static_cast<uint64_t>(kD) * 2;
+  // tensor maps of the K and V caches: [D, s_cap, Hkv, B], box 64 x 64 (one half tile)
   uint64_t kv_dims[4] = {static_cast<uint64_t>(kD), static_cast<uint64_t>(a.s_cap), static_cast<uint64_t>(Hkv),
                          static_cast<uint64_t>(B)};
   uint64_t kv_strides[3] = {static_cast<uint64_t>(a.kv_stride_s) * 2, static_cast<uint64_t>(a.kv_stride_h) * 2,
@@ -649,18 +735,13 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   if (Hkv == 1 && kv_strides[1] == 0) kv_strides[1] = kv_strides[0] * a.s_cap;  // a size-1 dimension never strides
   if (B == 1 && kv_strides[2] == 0) kv_strides[2] = kv_strides[1] * Hkv;
   const uint32_t kv_box[4] = {64, static_cast<uint32_t>(kBN), 1, 1};
-  uint64_t q_dims[4] = {static_cast<uint64_t>(kD), static_cast<uint64_t>(G), static_cast<uint64_t>(Hkv),
-                        static_cast<uint64_t>(a.tree.total_nodes)};
-  uint64_t q_strides[3] = {row_bytes, row_bytes * G, row_bytes * Hq};
-  const uint32_t q_box[4] = {64, static_cast<uint32_t>(G), 1, static_cast<uint32_t>(kBM / G)};
-  const CUtensorMap* tq = get_tmap(ctx, a.q, q_dims, q_strides, q_box);
   const CUtensorMap* tk = get_tmap(ctx, a.k_cache, kv_dims, kv_strides, kv_box);
   const CUtensorMap* tv = get_tmap(ctx, a.v_cache, kv_dims, kv_strides, kv_box);
-  if (!tq || !tk || !tv) {
+  if (!tk || !tv) {
     ctx->last_error = "cuTensorMapEncodeTiled failed";
     return FALCON_ERR_CUDA;
   }
-  const CUtensorMap mq = *tq, mk = *tk, mv = *tv;  // copies: later cache growth must not move what we pass
+  const CUtensorMap mk = *tk, mv = *tv;  // copies: later cache growth must not move what we pass
 
   const int max_tiles = (a.tree.max_prefix_len + a.tree.max_tree + kBN - 1) / kBN;
   int splits = a.n_splits;
@@ -679,6 +760,7 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   p.prefix_len = a.tree.prefix_len;
   p.status = a.tree.status;
   p.tree_mask = a.tree_mask;
+  p.q = static_cast<const __nv_bfloat16*>(a.q);
   p.out = static_cast<__nv_bfloat16*>(a.out);
 
   cudaLaunchConfig_t cfg = {};
@@ -693,7 +775,7 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   attr.val.clusterDim.z = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, mq, mk, mv, p);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, mk, mv, p);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tree_attn_tc_kernel launch");
   return FALCON_OK;
 }
