@@ -9,14 +9,15 @@
 // and every CTA normalises and stores its share of the rows.  No partial result
 // touches global memory.
 //
-// Inside a CTA (192 threads):
-//   warp 0    TMA producer: K and V tiles (bf16, 128-byte swizzle) into a 4-stage ring,
+// Inside a CTA (256 threads):
+//   warp 6    TMA producer: K and V tiles (bf16, 128-byte swizzle) into a 4-stage ring,
 //             completion on mbarriers; the first loads are issued before anything else.
-//   warp 1    one thread issues tcgen05.mma.  Both A operands live in tensor memory:
+//   warp 7    one elected lane issues tcgen05.mma (the whole warp runs the loop).  Both A operands live in tensor memory:
 //             S = Q.K^T (M=128, N=64, K=128) reads Q from TMEM and the K tile from shared
 //             memory; O += P.V (M=128, N=128, K=64) reads P from TMEM and the V tile from
 //             shared memory.  tcgen05.commit signals the consumers.
-//   warps 2-5 one thread per query row: loads its q row from global memory into TMEM once;
+//   warps 0-3 one thread per query row (warps 4-5 only pad the CTA so that the two service
+//             warps sit on other schedulers than the first two softmax warps): loads its q row from global memory into TMEM once;
 //             per tile tcgen05.ld of the score row, tree mask from the node's ancestor bit
 //             set, online softmax with a lazily updated maximum (the accumulator is
 //             rescaled only when the row maximum grows by more than 2^8), P written back
@@ -37,9 +38,12 @@ constexpr int kD = 128;
 constexpr int kBM = 128;          // query rows per CTA (TMEM lanes)
 constexpr int kBN = 64;           // keys per tile
 constexpr int kStages = 4;
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 256;    // warps 0-3 softmax (TMEM quadrant = warp), 4-5 idle, 6 producer, 7 MMA
+constexpr int kWarpProducer = 6;
+constexpr int kWarpMma = 7;
 constexpr int kMaxSplits = 8;
 constexpr uint32_t kSpinLimit = 1u << 18;
+constexpr uint32_t kSuspendHintNs = 2000;  // a waiting thread may sleep this long per try (it wakes when the phase completes)
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 constexpr uint32_t kTileBytes = kBN * kD * 2;      // 16 KB: two 64-column halves of 8 KB
@@ -105,9 +109,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
     uint32_t ok;
     asm volatile(
-        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3; selp.u32 %0, 1, 0, p; }"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
     if (ok) return true;
     if ((it & 255u) == 255u && *abort_flag) return false;
@@ -258,10 +262,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   // merge geometry: CTA `rank` owns rows [rank * rows_per, ...) of the tile
   const int rows_per = (n_valid + n_splits - 1) / n_splits;
 
-  if (warp == 0) {
+  const int n_sm_warps = (n_valid + 31) >> 5;  // softmax warps that own at least one query row
+  if (warp == kWarpProducer) {
     if (lane == 0) {
       s_abort = 0;
-      mbar_init(bar(kBarQ), 4);
+      mbar_init(bar(kBarQ), n_sm_warps);
       for (int s = 0; s < kStages; ++s) {
         mbar_init(bar(kBarKFull + s), 1);
         mbar_init(bar(kBarVFull + s), 1);
@@ -269,8 +274,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       }
       for (int s = 0; s < 2; ++s) {
         mbar_init(bar(kBarSFull + s), 1);
-        mbar_init(bar(kBarSEmpty + s), 4);
-        mbar_init(bar(kBarPFull + s), 4);
+        mbar_init(bar(kBarSEmpty + s), n_sm_warps);
+        mbar_init(bar(kBarPFull + s), n_sm_warps);
         mbar_init(bar(kBarPEmpty + s), 1);
       }
       mbar_init(bar(kBarODone), 1);
@@ -301,7 +306,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   // softmax threads fetch their q row while the rest sets up
   const int q4 = warp & 3;
   const int row = q4 * 32 + lane;
-  const bool is_sm = warp >= 2;
+  const bool is_sm = warp < 4;
   const bool valid = is_sm && row < n_valid;
   const bool warp_valid = is_sm && q4 * 32 < n_valid;
   uint4 qreg[16];
@@ -322,7 +327,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   tc_fence_after();
   const uint32_t tmem_base = s_tmem_base;
 
-  if (warp == 0) {
+  if (warp == kWarpProducer) {
     // ================================ TMA producer (ring refills) ================================
     if (lane == 0) {
       for (int j = kStages; j < n_my; ++j) {
@@ -339,49 +344,60 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         tma_load_4d(vdst + kHalfTile, &tm_v, bar(kBarVFull + st), 64, k0, kvh, b);
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == kWarpMma) {
     // ================================ MMA issuer ================================
-    if (lane == 0 && n_my > 0) {
-      bool ok = mbar_wait(bar(kBarQ), 0, abort_flag);
+    // The whole warp runs this loop (descriptors stay in uniform registers, which keeps the
+    // issue cost per tcgen05.mma low); one elected lane issues.
+    if (n_my > 0) {
+      uint32_t elected;
+      asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
+      bool ok = mbar_wait_warp(bar(kBarQ), 0, abort_flag);
       auto issue_pv = [&](int t) -> bool {
         const int st = t % kStages, pb = t & 1;
-        if (!mbar_wait(bar(kBarVFull + st), (t / kStages) & 1, abort_flag)) return false;
-        if (!mbar_wait(bar(kBarPFull + pb), (t >> 1) & 1, abort_flag)) return false;
+        if (!mbar_wait_warp(bar(kBarVFull + st), (t / kStages) & 1, abort_flag)) return false;
+        if (!mbar_wait_warp(bar(kBarPFull + pb), (t >> 1) & 1, abort_flag)) return false;
         tc_fence_after();
         const uint32_t vbase = smem_base + kOffKV + st * 2 * kTileBytes + kTileBytes;
+        if (elected) {
 #pragma unroll
-        for (int kk = 0; kk < kBN / 16; ++kk) {
-          // P: 16 keys = 8 packed columns; V: MN-major, 16 keys = 2 KB, the two 64-column halves 8 KB apart
-          const uint64_t bd = smem_desc(vbase + kk * 2048, kHalfTile, 1024);
-          umma_bf16_ts(tmem_base + kTmemO, tmem_base + kTmemP + pb * 32 + kk * 8, bd, kIdescPV,
-                       (t > 0 || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < kBN / 16; ++kk) {
+            // P: 16 keys = 8 packed columns; V: MN-major, 16 keys = 2 KB, the two 64-column halves 8 KB apart
+            const uint64_t bd = smem_desc(vbase + kk * 2048, kHalfTile, 1024);
+            umma_bf16_ts(tmem_base + kTmemO, tmem_base + kTmemP + pb * 32 + kk * 8, bd, kIdescPV,
+                         (t > 0 || kk > 0) ? 1u : 0u);
+          }
+          umma_commit(bar(kBarKVEmpty + st));
+          umma_commit(bar(kBarPEmpty + pb));
         }
-        umma_commit(bar(kBarKVEmpty + st));
-        umma_commit(bar(kBarPEmpty + pb));
+        __syncwarp();
         return true;
       };
       for (int j = 0; ok && j < n_my; ++j) {
         const int st = j % kStages, sb = j & 1;
-        if (!mbar_wait(bar(kBarKFull + st), (j / kStages) & 1, abort_flag)) { ok = false; break; }
-        if (j >= 2 && !mbar_wait(bar(kBarSEmpty + sb), ((j >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_wait_warp(bar(kBarKFull + st), (j / kStages) & 1, abort_flag)) { ok = false; break; }
+        if (j >= 2 && !mbar_wait_warp(bar(kBarSEmpty + sb), ((j >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t kbase = smem_base + kOffKV + st * 2 * kTileBytes;
+        if (elected) {
 #pragma unroll
-        for (int kk = 0; kk < kD / 16; ++kk) {
-          // K tile: K-major, 16 head-dim columns = 32 bytes inside the 128-byte swizzle row
-          const uint64_t bd = smem_desc(kbase + (kk >> 2) * kHalfTile + (kk & 3) * 32, 16, 1024);
-          umma_bf16_ts(tmem_base + kTmemS + sb * kBN, tmem_base + kTmemQ + kk * 8, bd, kIdescQK, kk > 0 ? 1u : 0u);
+          for (int kk = 0; kk < kD / 16; ++kk) {
+            // K tile: K-major, 16 head-dim columns = 32 bytes inside the 128-byte swizzle row
+            const uint64_t bd = smem_desc(kbase + (kk >> 2) * kHalfTile + (kk & 3) * 32, 16, 1024);
+            umma_bf16_ts(tmem_base + kTmemS + sb * kBN, tmem_base + kTmemQ + kk * 8, bd, kIdescQK, kk > 0 ? 1u : 0u);
+          }
+          umma_commit(bar(kBarSFull + sb));
         }
-        umma_commit(bar(kBarSFull + sb));
+        __syncwarp();
         if (j >= 1 && !issue_pv(j - 1)) { ok = false; break; }
       }
       if (ok) ok = issue_pv(n_my - 1);
-      umma_commit(bar(kBarODone));  // fires once every MMA issued so far has finished
+      if (elected) umma_commit(bar(kBarODone));  // fires once every MMA issued so far has finished
+      __syncwarp();
     }
-  } else {
-    // ================================ softmax / correction ================================
+  } else if (warp_valid) {
+    // ================================ softmax / correction (warps that own query rows) ================================
     const uint32_t tmem_lane = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16);
-    const int sm_tid = tid - 64;  // 0..127 over the four softmax warps
+    const int sm_tid = tid;  // softmax warps are warps 0..3
 
     // q row -> TMEM (bf16 pairs, 64 columns)
     if (warp_valid) {
@@ -438,7 +454,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         const int nv = S_valid - k0;  // 1..63 rows are real
         unsigned char* vtile = smem_gen + kOffKV + st * 2 * kTileBytes + kTileBytes;
         const int chunks = (kBN - nv) * 8;
-        for (int c = sm_tid; c < 2 * chunks; c += 128) {
+        for (int c = sm_tid; c < 2 * chunks; c += 32 * n_sm_warps) {
           const int half = c / chunks, cc = c % chunks;
           *reinterpret_cast<uint4*>(vtile + half * kHalfTile + nv * 128 + cc * 16) = make_uint4(0, 0, 0, 0);
         }
@@ -449,22 +465,39 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       float alpha = 1.f;
       bool need_rescale = false;
       if (valid) {
+        // scores stay raw; exp2(s * scale - m) is one FFMA + one MUFU per element (scale > 0 is
+        // guaranteed by the launcher, so the maximum can be taken on the raw scores)
         float s[64];
-        float tmax = -INFINITY;
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
         if (k0 + kBN <= Lc) {
 #pragma unroll
-          for (int c = 0; c < 64; ++c) {
-            s[c] = __uint_as_float(sr[c]) * scale;
-            tmax = fmaxf(tmax, s[c]);
+          for (int c = 0; c < 64; c += 4) {
+            s[c] = __uint_as_float(sr[c]);
+            s[c + 1] = __uint_as_float(sr[c + 1]);
+            s[c + 2] = __uint_as_float(sr[c + 2]);
+            s[c + 3] = __uint_as_float(sr[c + 3]);
+            mx0 = fmaxf(mx0, s[c]);
+            mx1 = fmaxf(mx1, s[c + 1]);
+            mx2 = fmaxf(mx2, s[c + 2]);
+            mx3 = fmaxf(mx3, s[c + 3]);
           }
         } else {
           const uint64_t vis = window64(anc_lo, anc_hi, k0 - Lc);
+          const uint32_t vlo = static_cast<uint32_t>(vis), vhi = static_cast<uint32_t>(vis >> 32);
 #pragma unroll
-          for (int c = 0; c < 64; ++c) {
-            s[c] = ((vis >> c) & 1ull) ? __uint_as_float(sr[c]) * scale : -INFINITY;
-            tmax = fmaxf(tmax, s[c]);
+          for (int c = 0; c < 64; c += 4) {
+            const uint32_t w = c < 32 ? vlo : vhi;
+            s[c] = ((w >> (c & 31)) & 1u) ? __uint_as_float(sr[c]) : -INFINITY;
+            s[c + 1] = ((w >> ((c + 1) & 31)) & 1u) ? __uint_as_float(sr[c + 1]) : -INFINITY;
+            s[c + 2] = ((w >> ((c + 2) & 31)) & 1u) ? __uint_as_float(sr[c + 2]) : -INFINITY;
+            s[c + 3] = ((w >> ((c + 3) & 31)) & 1u) ? __uint_as_float(sr[c + 3]) : -INFINITY;
+            mx0 = fmaxf(mx0, s[c]);
+            mx1 = fmaxf(mx1, s[c + 1]);
+            mx2 = fmaxf(mx2, s[c + 2]);
+            mx3 = fmaxf(mx3, s[c + 3]);
           }
         }
+        const float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale;  // -inf stays -inf
         if (m_used == -INFINITY) {
           m_used = tmax;  // nothing accumulated yet for this row (O and l are zero)
         } else if (tmax > m_used + kRescaleThreshold) {
@@ -473,17 +506,21 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           m_used = tmax;
           need_rescale = true;
         }
-        const float m_eff = (m_used == -INFINITY) ? 0.f : m_used;
-        float add0 = 0.f, add1 = 0.f;
+        const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+        float add0 = 0.f, add1 = 0.f, add2 = 0.f, add3 = 0.f;
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          const float p0 = ex2(s[2 * c] - m_eff), p1 = ex2(s[2 * c + 1] - m_eff);
+        for (int c = 0; c < 32; c += 2) {
+          const float p0 = ex2(fmaf(s[2 * c], scale, neg_m)), p1 = ex2(fmaf(s[2 * c + 1], scale, neg_m));
+          const float p2 = ex2(fmaf(s[2 * c + 2], scale, neg_m)), p3 = ex2(fmaf(s[2 * c + 3], scale, neg_m));
           add0 += p0;
           add1 += p1;
-          const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-          pk[c] = *reinterpret_cast<const uint32_t*>(&h);
+          add2 += p2;
+          add3 += p3;
+          const __nv_bfloat162 h0 = __floats2bfloat162_rn(p0, p1), h1 = __floats2bfloat162_rn(p2, p3);
+          pk[c] = *reinterpret_cast<const uint32_t*>(&h0);
+          pk[c + 1] = *reinterpret_cast<const uint32_t*>(&h1);
         }
-        l_sum += add0 + add1;
+        l_sum += (add0 + add1) + (add2 + add3);
       } else {
 #pragma unroll
         for (int c = 0; c < 32; ++c) pk[c] = 0u;
@@ -603,7 +640,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                                 c4 * 4) = *reinterpret_cast<const uint2*>(h);
     }
   }
-  if (warp == 0) {
+  if (warp == kWarpProducer) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
@@ -707,6 +744,7 @@ bool tree_attn_tc_supports(const falcon_ctx* ctx, const falcon_attn_args& a) {
   (void)ctx;
   if (a.head_dim != kD) return false;
   if (a.k_tree != nullptr) return false;
+  if (!(a.sm_scale > 0.f)) return false;  // the kernel takes row maxima on unscaled scores
   const int G = a.n_q_heads / a.n_kv_heads;
   if (!is_pow2(G) || G > kBM) return false;
   if (a.n_splits > kMaxSplits) return false;
