@@ -50,14 +50,18 @@ constexpr uint32_t kTileBytes = kBN * kD * 2;      // 16 KB: two 64-column halve
 constexpr uint32_t kHalfTile = kBN * 128;          // 8 KB
 constexpr uint32_t kOffKV = 0;
 constexpr uint32_t kKVBytes = kStages * 2 * kTileBytes;  // 128 KB
-// merge buffer: partial rows pushed by the cluster's CTAs, [split][row_local] rows of kMrgPitch floats
+// Merge: every CTA stages its partial rows in shared memory (over the K/V ring, which is idle by
+// then) and bulk-copies each owner's rows into that owner's merge buffer.  A row is kMrgPitch floats:
+// 128 accumulator columns, then the row's running maximum and sum.
 constexpr int kMrgRows = kBM + kMaxSplits;          // rows_per * n_splits <= n_valid + n_splits - 1
-constexpr int kMrgPitch = kD + 4;                   // 528-byte rows: 16-byte stores of 32 lanes spread over all banks
+constexpr int kMrgPitch = kD + 4;                   // 528-byte rows: 16-byte accesses of 32 lanes hit all banks evenly
+constexpr uint32_t kMrgRowBytes = kMrgPitch * 4;
+constexpr uint32_t kOffStage = kOffKV;              // [row][kMrgPitch] staging of this CTA's partial rows
 constexpr uint32_t kOffMrg = kOffKV + kKVBytes;
-constexpr uint32_t kMrgBytes = kMrgRows * kMrgPitch * 4;
-constexpr uint32_t kOffML = kOffMrg + kMrgBytes;    // float2 (max, sum) per merge row
-constexpr uint32_t kSmemBytes = kOffML + kMrgRows * 8;
+constexpr uint32_t kMrgBytes = kMrgRows * kMrgRowBytes;
+constexpr uint32_t kSmemBytes = kOffMrg + kMrgBytes;
 constexpr uint32_t kSmemAlloc = kSmemBytes + 1024;  // room to align the base to 1 KB
+static_assert(kBM * kMrgRowBytes <= kKVBytes, "staging must fit in the K/V ring");
 
 // tensor memory columns (32-bit each, 128 lanes)
 constexpr uint32_t kTmemCols = 512;
@@ -76,7 +80,8 @@ enum {
   kBarPFull = kBarSEmpty + 2,        // [2]
   kBarPEmpty = kBarPFull + 2,        // [2]  also "P.V of tile j finished"
   kBarODone = kBarPEmpty + 2,
-  kNumBars = kBarODone + 1
+  kBarMrg = kBarODone + 1,           // all partial rows this CTA owns have arrived
+  kNumBars = kBarMrg + 1
 };
 
 struct TcParams {
@@ -192,21 +197,21 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
   return r;
 }
-__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float a, float b, float c, float d) {
-  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
+// Asynchronous copy of `bytes` (multiple of 16) from this CTA's shared memory into a cluster peer's;
+// completion is counted on the peer's mbarrier.
+__device__ __forceinline__ void bulk_copy_to_peer(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes,
+                                                  uint32_t bar_cluster) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   dst_cluster),
+               "r"(src_cta), "r"(bytes), "r"(bar_cluster)
                : "memory");
-}
-__device__ __forceinline__ void st_cluster_v2(uint32_t addr, float a, float b) {
-  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
 }
 
 // 64 visibility bits for tree indices off .. off+63 of a 128-bit set; negative indices (prefix keys) are visible.
@@ -279,7 +284,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         mbar_init(bar(kBarPEmpty + s), 1);
       }
       mbar_init(bar(kBarODone), 1);
+      mbar_init(bar(kBarMrg), 1);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      if (n_splits > 1) {
+        // this CTA will receive rows_mine rows from every split (its own included)
+        const int r0 = split * rows_per;
+        const int mine = max(0, min(n_valid, r0 + rows_per) - r0);
+        mbar_expect_tx(bar(kBarMrg), static_cast<uint32_t>(n_splits * mine) * kMrgRowBytes);
+      }
       // first ring fill right away: these loads need nothing but the barriers this thread just made
       const int pre = min(n_my, kStages);
       for (int j = 0; j < pre; ++j) {
@@ -326,6 +338,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = s_tmem_base;
+  // Cluster phase 1: "my merge barrier exists".  Arrive now, wait just before the first remote copy.
+  if (n_splits > 1) cluster_arrive();
 
   if (warp == kWarpProducer) {
     // ================================ TMA producer (ring refills) ================================
@@ -553,55 +567,53 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       if (lane == 0) mbar_arrive(bar(kBarPFull + sb));
     }
 
-    // ---- this split's partial rows: straight to global (one split) or pushed to their owner ----
+    // ---- this split's partial rows: straight to global (one split) or staged for the merge ----
     bool have = (n_my > 0) && !*abort_flag;
     if (have) have = mbar_wait_warp(bar(kBarODone), 0, abort_flag);
     tc_fence_after();
-    if (warp_valid) {
-      const bool write = have && valid;
-      if (n_splits == 1) {
-        const float inv = (write && l_sum > 0.f) ? 1.f / l_sum : 0.f;
-        const int mg = mtile * kBM + row;
-        __nv_bfloat16* dst = p.out + (static_cast<int64_t>(node_base + mg / G) * p.Hq + kvh * G + mg % G) * kD;
+    const bool write = have && valid;
+    if (n_splits == 1) {
+      const float inv = (write && l_sum > 0.f) ? 1.f / l_sum : 0.f;
+      const int mg = mtile * kBM + row;
+      __nv_bfloat16* dst = p.out + (static_cast<int64_t>(node_base + mg / G) * p.Hq + kvh * G + mg % G) * kD;
 #pragma unroll 1
-        for (int ch = 0; ch < 4; ++ch) {
-          uint32_t o[32];
-          FALCON_TMEM_LD32(tmem_lane + kTmemO + ch * 32, o);
-          tmem_wait_ld();
-          if (valid) {
+      for (int ch = 0; ch < 2; ++ch) {
+        uint32_t o[64];
+        FALCON_TMEM_LD32(tmem_lane + kTmemO + ch * 64, o);
+        FALCON_TMEM_LD32(tmem_lane + kTmemO + ch * 64 + 32, (o + 32));
+        tmem_wait_ld();
+        if (valid) {
 #pragma unroll
-            for (int c8 = 0; c8 < 4; ++c8) {
-              __align__(16) __nv_bfloat162 h[4];
+          for (int c8 = 0; c8 < 8; ++c8) {
+            __align__(16) __nv_bfloat162 h[4];
 #pragma unroll
-              for (int c = 0; c < 4; ++c)
-                h[c] = __floats2bfloat162_rn(__uint_as_float(o[8 * c8 + 2 * c]) * inv,
-                                             __uint_as_float(o[8 * c8 + 2 * c + 1]) * inv);
-              *reinterpret_cast<uint4*>(dst + ch * 32 + c8 * 8) = *reinterpret_cast<const uint4*>(h);
-            }
-          }
-        }
-      } else {
-        const int owner = valid ? row / rows_per : 0;
-        const int slot = split * rows_per + (valid ? row % rows_per : 0);
-        const uint32_t dst = map_to_rank(smem_base + kOffMrg + static_cast<uint32_t>(slot) * (kMrgPitch * 4), owner);
-        if (valid)
-          st_cluster_v2(map_to_rank(smem_base + kOffML + static_cast<uint32_t>(slot) * 8, owner),
-                        write ? m_used : -INFINITY, write ? l_sum : 0.f);
-        if (have) {
-#pragma unroll 1
-          for (int ch = 0; ch < 4; ++ch) {
-            uint32_t o[32];
-            FALCON_TMEM_LD32(tmem_lane + kTmemO + ch * 32, o);
-            tmem_wait_ld();
-            if (valid) {
-#pragma unroll
-              for (int c4 = 0; c4 < 8; ++c4)
-                st_cluster_v4(dst + (ch * 32 + c4 * 4) * 4, __uint_as_float(o[4 * c4]), __uint_as_float(o[4 * c4 + 1]),
-                              __uint_as_float(o[4 * c4 + 2]), __uint_as_float(o[4 * c4 + 3]));
-            }
+            for (int c = 0; c < 4; ++c)
+              h[c] = __floats2bfloat162_rn(__uint_as_float(o[8 * c8 + 2 * c]) * inv,
+                                           __uint_as_float(o[8 * c8 + 2 * c + 1]) * inv);
+            *reinterpret_cast<uint4*>(dst + ch * 64 + c8 * 8) = *reinterpret_cast<const uint4*>(h);
           }
         }
       }
+    } else {
+      // the K/V ring is idle now (all of this CTA's MMAs have finished): stage row -> [row][kMrgPitch]
+      float* stage = reinterpret_cast<float*>(smem_gen + kOffStage) + row * kMrgPitch;
+      if (have) {
+#pragma unroll 1
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t o[64];
+          FALCON_TMEM_LD32(tmem_lane + kTmemO + ch * 64, o);
+          FALCON_TMEM_LD32(tmem_lane + kTmemO + ch * 64 + 32, (o + 32));
+          tmem_wait_ld();
+          if (valid) {
+#pragma unroll
+            for (int c4 = 0; c4 < 16; ++c4)
+              *reinterpret_cast<uint4*>(stage + ch * 64 + c4 * 4) =
+                  make_uint4(o[4 * c4], o[4 * c4 + 1], o[4 * c4 + 2], o[4 * c4 + 3]);
+          }
+        }
+      }
+      if (valid) *reinterpret_cast<float2*>(stage + kD) = make_float2(write ? m_used : -INFINITY, write ? l_sum : 0.f);
+      fence_async_smem();  // the bulk copies below read these rows through the async proxy
     }
   }
 
@@ -610,22 +622,35 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   __syncthreads();
   if (s_abort && tid == 0) dev_status_or(p.status, b, FALCON_DEV_TIMEOUT);
   if (n_splits > 1) {
-    cluster_sync_all();  // every CTA's rows have landed in their owner's shared memory
+    cluster_wait();  // phase 1 done: every peer's merge barrier is initialised
+    if (warp == kWarpProducer && lane == 0) {
+      // one bulk copy per owner: its rows of this split, contiguous in the staging area
+      for (int o = 0; o < n_splits; ++o) {
+        const int r0 = o * rows_per;
+        const int cnt = min(n_valid, r0 + rows_per) - r0;
+        if (cnt <= 0) break;
+        bulk_copy_to_peer(map_to_rank(smem_base + kOffMrg + static_cast<uint32_t>(split * rows_per) * kMrgRowBytes, o),
+                          smem_base + kOffStage + static_cast<uint32_t>(r0) * kMrgRowBytes,
+                          static_cast<uint32_t>(cnt) * kMrgRowBytes, map_to_rank(bar(kBarMrg), o));
+      }
+    }
+    __syncwarp();
     const int row0 = split * rows_per;
     const int rows_mine = max(0, min(n_valid, row0 + rows_per) - row0);
+    const bool got = rows_mine == 0 || mbar_wait_warp(bar(kBarMrg), 0, abort_flag);
     const float* mrg = reinterpret_cast<const float*>(smem_gen + kOffMrg);
-    const float2* ml = reinterpret_cast<const float2*>(smem_gen + kOffML);
-    for (int item = tid; item < rows_mine * (kD / 4); item += kTcThreads) {
+    for (int item = tid; got && item < rows_mine * (kD / 4); item += kTcThreads) {
       const int rl = item / (kD / 4), c4 = item % (kD / 4);
       float gm = -INFINITY;
-      for (int s = 0; s < n_splits; ++s) gm = fmaxf(gm, ml[s * rows_per + rl].x);
+      for (int s = 0; s < n_splits; ++s) gm = fmaxf(gm, mrg[(s * rows_per + rl) * kMrgPitch + kD]);
       float lsum = 0.f, a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
       for (int s = 0; s < n_splits; ++s) {
-        const float2 m_l = ml[s * rows_per + rl];
-        if (m_l.x == -INFINITY) continue;
+        const float* rowp = mrg + (s * rows_per + rl) * kMrgPitch;
+        const float2 m_l = *reinterpret_cast<const float2*>(rowp + kD);
+        if (m_l.x == -INFINITY) continue;  // that split saw no key of this row: its columns are not valid
         const float w = ex2(m_l.x - gm);
         lsum = fmaf(m_l.y, w, lsum);
-        const float4 x = *reinterpret_cast<const float4*>(mrg + (s * rows_per + rl) * kMrgPitch + c4 * 4);
+        const float4 x = *reinterpret_cast<const float4*>(rowp + c4 * 4);
         a0 = fmaf(x.x, w, a0);
         a1 = fmaf(x.y, w, a1);
         a2 = fmaf(x.z, w, a2);
@@ -639,6 +664,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       *reinterpret_cast<uint2*>(p.out + (static_cast<int64_t>(node_base + mg / G) * p.Hq + kvh * G + mg % G) * kD +
                                 c4 * 4) = *reinterpret_cast<const uint2*>(h);
     }
+    // Cluster phase 2: nobody leaves while a peer may still be reading its staging rows or
+    // writing into its merge buffer (an owner arrives only after all its rows have landed).
+    cluster_arrive();
+    cluster_wait();
   }
   if (warp == kWarpProducer) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
