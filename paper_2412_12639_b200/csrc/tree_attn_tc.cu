@@ -10,14 +10,13 @@
 // touches global memory.
 //
 // Inside a CTA (256 threads):
-//   warp 6    TMA producer: K and V tiles (bf16, 128-byte swizzle) into a 4-stage ring,
-//             completion on mbarriers; the first loads are issued before anything else.
-//   warp 7    one elected lane issues tcgen05.mma (the whole warp runs the loop).  Both A operands live in tensor memory:
-//             S = Q.K^T (M=128, N=64, K=128) reads Q from TMEM and the K tile from shared
-//             memory; O += P.V (M=128, N=128, K=64) reads P from TMEM and the V tile from
+//   warp 6    TMA producer: the Q tile first, then K and V tiles (bf16, 128-byte swizzle) into a
+//             3-stage ring, completion on mbarriers; the first loads are issued before anything else.
+//   warp 7    one elected lane issues tcgen05.mma (the whole warp runs the loop).  
+//             S = Q.K^T (M=128, N=64, K=128) reads Q and the K tile from shared memory; O += P.V (M=128, N=128, K=64) reads P from TMEM and the V tile from
 //             shared memory.  tcgen05.commit signals the consumers.
 //   warps 0-3 one thread per query row (warps 4-5 only pad the CTA so that the two service
-//             warps sit on other schedulers than the first two softmax warps): loads its q row from global memory into TMEM once;
+//             warps sit on other schedulers than the first two softmax warps):
 //             per tile tcgen05.ld of the score row, tree mask from the node's ancestor bit
 //             set, online softmax with a lazily updated maximum (the accumulator is
 //             rescaled only when the row maximum grows by more than 2^8), P written back
@@ -31,13 +30,18 @@
 
 #include "common.cuh"
 
+// Profiling hook, off by default: a build may predefine it to record per-phase time stamps.
+#ifndef FALCON_TRACE
+#define FALCON_TRACE(who, id)
+#endif
+
 namespace falcon {
 namespace {
 
 constexpr int kD = 128;
 constexpr int kBM = 128;          // query rows per CTA (TMEM lanes)
 constexpr int kBN = 64;           // keys per tile
-constexpr int kStages = 4;
+constexpr int kStages = 3;
 constexpr int kTcThreads = 256;    // warps 0-3 softmax (TMEM quadrant = warp), 4-5 idle, 6 producer, 7 MMA
 constexpr int kWarpProducer = 6;
 constexpr int kWarpMma = 7;
@@ -48,30 +52,31 @@ constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 constexpr uint32_t kTileBytes = kBN * kD * 2;      // 16 KB: two 64-column halves of 8 KB
 constexpr uint32_t kHalfTile = kBN * 128;          // 8 KB
-constexpr uint32_t kOffKV = 0;
-constexpr uint32_t kKVBytes = kStages * 2 * kTileBytes;  // 128 KB
-// Merge: every CTA stages its partial rows in shared memory (over the K/V ring, which is idle by
+constexpr uint32_t kQBytes = kBM * kD * 2;          // 32 KB: two 64-column halves of 16 KB
+constexpr uint32_t kOffQ = 0;
+constexpr uint32_t kOffKV = kOffQ + kQBytes;
+constexpr uint32_t kKVBytes = kStages * 2 * kTileBytes;  // 96 KB
+// Merge: every CTA stages its partial rows in shared memory (over Q and the K/V ring, idle by
 // then) and bulk-copies each owner's rows into that owner's merge buffer.  A row is kMrgPitch floats:
 // 128 accumulator columns, then the row's running maximum and sum.
 constexpr int kMrgRows = kBM + kMaxSplits;          // rows_per * n_splits <= n_valid + n_splits - 1
 constexpr int kMrgPitch = kD + 4;                   // 528-byte rows: 16-byte accesses of 32 lanes hit all banks evenly
 constexpr uint32_t kMrgRowBytes = kMrgPitch * 4;
-constexpr uint32_t kOffStage = kOffKV;              // [row][kMrgPitch] staging of this CTA's partial rows
+constexpr uint32_t kOffStage = kOffQ;               // [row][kMrgPitch] staging of this CTA's partial rows
 constexpr uint32_t kOffMrg = kOffKV + kKVBytes;
 constexpr uint32_t kMrgBytes = kMrgRows * kMrgRowBytes;
 constexpr uint32_t kSmemBytes = kOffMrg + kMrgBytes;
 constexpr uint32_t kSmemAlloc = kSmemBytes + 1024;  // room to align the base to 1 KB
-static_assert(kBM * kMrgRowBytes <= kKVBytes, "staging must fit in the K/V ring");
+static_assert(kBM * kMrgRowBytes <= kQBytes + kKVBytes, "staging must fit over Q and the K/V ring");
 
 // tensor memory columns (32-bit each, 128 lanes)
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemO = 0;      // 128 columns: fp32 accumulator
 constexpr uint32_t kTmemS = 128;    // 2 x 64 columns: fp32 scores
 constexpr uint32_t kTmemP = 256;    // 2 x 32 columns: bf16 pairs
-constexpr uint32_t kTmemQ = 320;    // 64 columns: bf16 pairs
 
 enum {
-  kBarQ = 0,                         // q rows are in TMEM (4 warps)
+  kBarQ = 0,                         // the Q tile has landed in shared memory
   kBarKFull = 1,                     // [kStages]
   kBarVFull = kBarKFull + kStages,   // [kStages]
   kBarKVEmpty = kBarVFull + kStages, // [kStages]
@@ -148,6 +153,14 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// D[tmem] (+)= A[smem] . B[smem]
+__device__ __forceinline__ void umma_bf16_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 // D[tmem] (+)= A[tmem] . B[smem]
 __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                              uint32_t accumulate) {
@@ -198,6 +211,11 @@ __device__ __forceinline__ float ex2(float x) {
 }
 
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+// Arrival that orders nothing: used where the barrier only keeps CTAs alive, so that it does not
+// have to wait for this thread's outstanding global stores.
+__device__ __forceinline__ void cluster_arrive_relaxed() {
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {
   uint32_t r;
@@ -227,19 +245,21 @@ __device__ __forceinline__ uint64_t window64(uint64_t lo, uint64_t hi, int off) 
 
 // ------------------------------------------------------------------------------------ kernel
 __global__ void __launch_bounds__(kTcThreads, 1)
-tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                    const TcParams p) {
+tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                    const __grid_constant__ CUtensorMap tm_v, const TcParams p) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t s_bars[kNumBars];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  FALCON_TRACE(tid == 0, 0);
   const int n_splits = gridDim.x, split = blockIdx.x;  // cluster = all CTAs of a row of the grid
   const int kvh = blockIdx.y % p.Hkv, mtile = blockIdx.y / p.Hkv, b = blockIdx.z;
   const int G = p.G;
 
   if (tid == 0) {
+    prefetch_tmap(&tm_q);
     prefetch_tmap(&tm_k);
     prefetch_tmap(&tm_v);
   }
@@ -270,8 +290,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   const int n_sm_warps = (n_valid + 31) >> 5;  // softmax warps that own at least one query row
   if (warp == kWarpProducer) {
     if (lane == 0) {
+      FALCON_TRACE(true, 1);
       s_abort = 0;
-      mbar_init(bar(kBarQ), n_sm_warps);
+      mbar_init(bar(kBarQ), 1);
       for (int s = 0; s < kStages; ++s) {
         mbar_init(bar(kBarKFull + s), 1);
         mbar_init(bar(kBarVFull + s), 1);
@@ -292,7 +313,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         const int mine = max(0, min(n_valid, r0 + rows_per) - r0);
         mbar_expect_tx(bar(kBarMrg), static_cast<uint32_t>(n_splits * mine) * kMrgRowBytes);
       }
-      // first ring fill right away: these loads need nothing but the barriers this thread just made
+      // first loads right away (they need nothing but the barriers this thread just made), Q in front
+      // so that it is not queued behind the K/V tiles
+      if (n_my > 0) {
+        const int node0 = node_base + mtile * (kBM / G);
+        mbar_expect_tx(bar(kBarQ), kQBytes);
+        tma_load_4d(smem_base + kOffQ, &tm_q, bar(kBarQ), 0, 0, kvh, node0);
+        tma_load_4d(smem_base + kOffQ + kQBytes / 2, &tm_q, bar(kBarQ), 64, 0, kvh, node0);
+      }
       const int pre = min(n_my, kStages);
       for (int j = 0; j < pre; ++j) {
         const int k0 = (t_begin + j) * kBN;
@@ -305,6 +333,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         tma_load_4d(vdst, &tm_v, bar(kBarVFull + j), 0, k0, kvh, b);
         tma_load_4d(vdst + kHalfTile, &tm_v, bar(kBarVFull + j), 64, k0, kvh, b);
       }
+      FALCON_TRACE(true, 2);
       if (split == 0 && mtile == 0 && kvh == 0 && (L + T > p.s_cap || T_real > FALCON_T_MAX))
         dev_status_or(p.status, b, FALCON_DEV_CAPACITY);
     }
@@ -315,29 +344,17 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
 
-  // softmax threads fetch their q row while the rest sets up
   const int q4 = warp & 3;
   const int row = q4 * 32 + lane;
   const bool is_sm = warp < 4;
   const bool valid = is_sm && row < n_valid;
   const bool warp_valid = is_sm && q4 * 32 < n_valid;
-  uint4 qreg[16];
-  if (warp_valid) {
-#pragma unroll
-    for (int i = 0; i < 16; ++i) qreg[i] = make_uint4(0, 0, 0, 0);
-    if (valid) {
-      const int mg = mtile * kBM + row;
-      const uint4* src = reinterpret_cast<const uint4*>(
-          p.q + (static_cast<int64_t>(node_base + mg / G) * p.Hq + kvh * G + mg % G) * kD);
-#pragma unroll
-      for (int i = 0; i < 16; ++i) qreg[i] = __ldg(src + i);
-    }
-  }
 
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = s_tmem_base;
+  FALCON_TRACE(tid == 0, 4);
   // Cluster phase 1: "my merge barrier exists".  Arrive now, wait just before the first remote copy.
   if (n_splits > 1) cluster_arrive();
 
@@ -366,10 +383,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       uint32_t elected;
       asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
       bool ok = mbar_wait_warp(bar(kBarQ), 0, abort_flag);
+      FALCON_TRACE(elected, 5);
       auto issue_pv = [&](int t) -> bool {
         const int st = t % kStages, pb = t & 1;
         if (!mbar_wait_warp(bar(kBarVFull + st), (t / kStages) & 1, abort_flag)) return false;
         if (!mbar_wait_warp(bar(kBarPFull + pb), (t >> 1) & 1, abort_flag)) return false;
+        FALCON_TRACE(elected && t < 6, 12 + 4 * t);
         tc_fence_after();
         const uint32_t vbase = smem_base + kOffKV + st * 2 * kTileBytes + kTileBytes;
         if (elected) {
@@ -382,6 +401,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
           }
           umma_commit(bar(kBarKVEmpty + st));
           umma_commit(bar(kBarPEmpty + pb));
+          FALCON_TRACE(t < 6, 13 + 4 * t);
         }
         __syncwarp();
         return true;
@@ -390,16 +410,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         const int st = j % kStages, sb = j & 1;
         if (!mbar_wait_warp(bar(kBarKFull + st), (j / kStages) & 1, abort_flag)) { ok = false; break; }
         if (j >= 2 && !mbar_wait_warp(bar(kBarSEmpty + sb), ((j >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+        FALCON_TRACE(elected && j < 6, 10 + 4 * j);
         tc_fence_after();
         const uint32_t kbase = smem_base + kOffKV + st * 2 * kTileBytes;
         if (elected) {
 #pragma unroll
           for (int kk = 0; kk < kD / 16; ++kk) {
-            // K tile: K-major, 16 head-dim columns = 32 bytes inside the 128-byte swizzle row
+            // Q and K tiles: K-major, 16 head-dim columns = 32 bytes inside the 128-byte swizzle row
+            const uint64_t ad = smem_desc(smem_base + kOffQ + (kk >> 2) * (kQBytes / 2) + (kk & 3) * 32, 16, 1024);
             const uint64_t bd = smem_desc(kbase + (kk >> 2) * kHalfTile + (kk & 3) * 32, 16, 1024);
-            umma_bf16_ts(tmem_base + kTmemS + sb * kBN, tmem_base + kTmemQ + kk * 8, bd, kIdescQK, kk > 0 ? 1u : 0u);
+            umma_bf16_ss(tmem_base + kTmemS + sb * kBN, ad, bd, kIdescQK, kk > 0 ? 1u : 0u);
           }
           umma_commit(bar(kBarSFull + sb));
+          FALCON_TRACE(j < 6, 11 + 4 * j);
         }
         __syncwarp();
         if (j >= 1 && !issue_pv(j - 1)) { ok = false; break; }
@@ -412,17 +435,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     // ================================ softmax / correction (warps that own query rows) ================================
     const uint32_t tmem_lane = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16);
     const int sm_tid = tid;  // softmax warps are warps 0..3
-
-    // q row -> TMEM (bf16 pairs, 64 columns)
-    if (warp_valid) {
-      const uint32_t* qw = reinterpret_cast<const uint32_t*>(qreg);
-      FALCON_TMEM_ST32(tmem_lane + kTmemQ, qw);
-      FALCON_TMEM_ST32(tmem_lane + kTmemQ + 32, (qw + 32));
-      tmem_wait_st();
-    }
-    tc_fence_before();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(bar(kBarQ));
 
     uint64_t anc_lo = 0, anc_hi = 0;
     if (valid) {
@@ -451,6 +463,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       const int sb = j & 1, u2 = j >> 1, st = j % kStages;
       const int k0 = (t_begin + j) * kBN;
       if (!mbar_wait_warp(bar(kBarSFull + sb), u2 & 1, abort_flag)) break;
+      FALCON_TRACE(tid == 0 && j < 6, 40 + 4 * j);
       tc_fence_after();
       uint32_t sr[64];
       if (warp_valid) {
@@ -461,6 +474,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(kBarSEmpty + sb));
+      FALCON_TRACE(tid == 0 && j < 6, 41 + 4 * j);
 
       // the sequence's last tile: rows of V past the last key may hold anything (0 x NaN = NaN in the MMA)
       if (k0 + kBN > S_valid) {
@@ -540,6 +554,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         for (int c = 0; c < 32; ++c) pk[c] = 0u;
       }
 
+      FALCON_TRACE(tid == 0 && j < 6, 42 + 4 * j);
       // P buffer free again?  (P.V of tile j-2 finished)
       if (u2 >= 1 && !mbar_wait_warp(bar(kBarPEmpty + sb), (u2 - 1) & 1, abort_flag)) break;
 
@@ -565,11 +580,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(kBarPFull + sb));
+      FALCON_TRACE(tid == 0 && j < 6, 43 + 4 * j);
     }
 
     // ---- this split's partial rows: straight to global (one split) or staged for the merge ----
     bool have = (n_my > 0) && !*abort_flag;
     if (have) have = mbar_wait_warp(bar(kBarODone), 0, abort_flag);
+    FALCON_TRACE(tid == 0, 70);
     tc_fence_after();
     const bool write = have && valid;
     if (n_splits == 1) {
@@ -617,12 +634,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     }
   }
 
+  FALCON_TRACE(tid == 0, 71);
   // ================================ cluster merge ================================
   tc_fence_before();
   __syncthreads();
+  FALCON_TRACE(tid == 0, 72);
   if (s_abort && tid == 0) dev_status_or(p.status, b, FALCON_DEV_TIMEOUT);
   if (n_splits > 1) {
     cluster_wait();  // phase 1 done: every peer's merge barrier is initialised
+    FALCON_TRACE(tid == 0, 73);
     if (warp == kWarpProducer && lane == 0) {
       // one bulk copy per owner: its rows of this split, contiguous in the staging area
       for (int o = 0; o < n_splits; ++o) {
@@ -638,23 +658,37 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     const int row0 = split * rows_per;
     const int rows_mine = max(0, min(n_valid, row0 + rows_per) - row0);
     const bool got = rows_mine == 0 || mbar_wait_warp(bar(kBarMrg), 0, abort_flag);
+    FALCON_TRACE(tid == 0, 74);
     const float* mrg = reinterpret_cast<const float*>(smem_gen + kOffMrg);
     for (int item = tid; got && item < rows_mine * (kD / 4); item += kTcThreads) {
       const int rl = item / (kD / 4), c4 = item % (kD / 4);
+      // all loads first (independent), then the arithmetic
+      float2 m_l[kMaxSplits];
+      float4 x[kMaxSplits];
+#pragma unroll
+      for (int s = 0; s < kMaxSplits; ++s) {
+        m_l[s] = make_float2(-INFINITY, 0.f);
+        x[s] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (s < n_splits) {
+          const float* rowp = mrg + (s * rows_per + rl) * kMrgPitch;
+          m_l[s] = *reinterpret_cast<const float2*>(rowp + kD);
+          x[s] = *reinterpret_cast<const float4*>(rowp + c4 * 4);
+        }
+      }
       float gm = -INFINITY;
-      for (int s = 0; s < n_splits; ++s) gm = fmaxf(gm, mrg[(s * rows_per + rl) * kMrgPitch + kD]);
+#pragma unroll
+      for (int s = 0; s < kMaxSplits; ++s) gm = fmaxf(gm, m_l[s].x);
       float lsum = 0.f, a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-      for (int s = 0; s < n_splits; ++s) {
-        const float* rowp = mrg + (s * rows_per + rl) * kMrgPitch;
-        const float2 m_l = *reinterpret_cast<const float2*>(rowp + kD);
-        if (m_l.x == -INFINITY) continue;  // that split saw no key of this row: its columns are not valid
-        const float w = ex2(m_l.x - gm);
-        lsum = fmaf(m_l.y, w, lsum);
-        const float4 x = *reinterpret_cast<const float4*>(rowp + c4 * 4);
-        a0 = fmaf(x.x, w, a0);
-        a1 = fmaf(x.y, w, a1);
-        a2 = fmaf(x.z, w, a2);
-        a3 = fmaf(x.w, w, a3);
+#pragma unroll
+      for (int s = 0; s < kMaxSplits; ++s) {
+        if (m_l[s].x != -INFINITY) {  // a split that saw no key of this row has no valid columns
+          const float w = ex2(m_l[s].x - gm);
+          lsum = fmaf(m_l[s].y, w, lsum);
+          a0 = fmaf(x[s].x, w, a0);
+          a1 = fmaf(x[s].y, w, a1);
+          a2 = fmaf(x[s].z, w, a2);
+          a3 = fmaf(x[s].w, w, a3);
+        }
       }
       const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
       const int mg = mtile * kBM + row0 + rl;
@@ -666,8 +700,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     }
     // Cluster phase 2: nobody leaves while a peer may still be reading its staging rows or
     // writing into its merge buffer (an owner arrives only after all its rows have landed).
-    cluster_arrive();
+    FALCON_TRACE(tid == 0, 75);
+    cluster_arrive_relaxed();
     cluster_wait();
+    FALCON_TRACE(tid == 0, 76);
   }
   if (warp == kWarpProducer) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
@@ -802,13 +838,20 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   if (Hkv == 1 && kv_strides[1] == 0) kv_strides[1] = kv_strides[0] * a.s_cap;  // a size-1 dimension never strides
   if (B == 1 && kv_strides[2] == 0) kv_strides[2] = kv_strides[1] * Hkv;
   const uint32_t kv_box[4] = {64, static_cast<uint32_t>(kBN), 1, 1};
+  // q [D, G, Hkv, N]: one box is the 128 query rows (128/G nodes x G heads) of a KV head, half of D
+  const uint64_t row_bytes = static_cast<uint64_t>(kD) * 2;
+  uint64_t q_dims[4] = {static_cast<uint64_t>(kD), static_cast<uint64_t>(G), static_cast<uint64_t>(Hkv),
+                        static_cast<uint64_t>(a.tree.total_nodes)};
+  uint64_t q_strides[3] = {row_bytes, row_bytes * G, row_bytes * Hq};
+  const uint32_t q_box[4] = {64, static_cast<uint32_t>(G), 1, static_cast<uint32_t>(kBM / G)};
+  const CUtensorMap* tq = get_tmap(ctx, a.q, q_dims, q_strides, q_box);
   const CUtensorMap* tk = get_tmap(ctx, a.k_cache, kv_dims, kv_strides, kv_box);
   const CUtensorMap* tv = get_tmap(ctx, a.v_cache, kv_dims, kv_strides, kv_box);
-  if (!tk || !tv) {
+  if (!tq || !tk || !tv) {
     ctx->last_error = "cuTensorMapEncodeTiled failed";
     return FALCON_ERR_CUDA;
   }
-  const CUtensorMap mk = *tk, mv = *tv;  // copies: later cache growth must not move what we pass
+  const CUtensorMap mq = *tq, mk = *tk, mv = *tv;  // copies: later cache growth must not move what we pass
 
   const int max_tiles = (a.tree.max_prefix_len + a.tree.max_tree + kBN - 1) / kBN;
   int splits = a.n_splits;
@@ -842,7 +885,7 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   attr.val.clusterDim.z = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, mk, mv, p);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, mq, mk, mv, p);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tree_attn_tc_kernel launch");
   return FALCON_OK;
 }
