@@ -11,7 +11,7 @@
 //
 // Inside a CTA (256 threads):
 //   warp 6    TMA producer: the Q tile first, then K and V tiles (bf16, 128-byte swizzle) into a
-//             3-stage ring, completion on mbarriers; the first loads are issued before anything else.
+//             5-stage ring, completion on mbarriers; the first loads are issued before anything else.
 //   warp 7    one elected lane issues tcgen05.mma (the whole warp runs the loop).  
 //             S = Q.K^T (M=128, N=64, K=128) reads Q and the K tile from shared memory; O += P.V (M=128, N=128, K=64) reads P from TMEM and the V tile from
 //             shared memory.  tcgen05.commit signals the consumers.
@@ -41,13 +41,20 @@ namespace {
 constexpr int kD = 128;
 constexpr int kBM = 128;          // query rows per CTA (TMEM lanes)
 constexpr int kBN = 64;           // keys per tile
-constexpr int kStages = 3;
+constexpr int kStages = 5;
+#ifndef EXP_PREFETCH
+#define EXP_PREFETCH 5
+#endif
+constexpr int kPrefetch = EXP_PREFETCH;  // tiles requested ahead of the consumer (<= kStages)
 constexpr int kTcThreads = 256;    // warps 0-3 softmax (TMEM quadrant = warp), 4-5 idle, 6 producer, 7 MMA
 constexpr int kWarpProducer = 6;
 constexpr int kWarpMma = 7;
 constexpr int kMaxSplits = 8;
 constexpr uint32_t kSpinLimit = 1u << 18;
-constexpr uint32_t kSuspendHintNs = 2000;  // a waiting thread may sleep this long per try (it wakes when the phase completes)
+#ifndef EXP_HINT
+#define EXP_HINT 2000
+#endif
+constexpr uint32_t kSuspendHintNs = EXP_HINT;  // a waiting thread may sleep this long per try (it wakes when the phase completes)
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 constexpr uint32_t kTileBytes = kBN * kD * 2;      // 16 KB: two 64-column halves of 8 KB
@@ -55,19 +62,20 @@ constexpr uint32_t kHalfTile = kBN * 128;          // 8 KB
 constexpr uint32_t kQBytes = kBM * kD * 2;          // 32 KB: two 64-column halves of 16 KB
 constexpr uint32_t kOffQ = 0;
 constexpr uint32_t kOffKV = kOffQ + kQBytes;
-constexpr uint32_t kKVBytes = kStages * 2 * kTileBytes;  // 96 KB
-// Merge: every CTA stages its partial rows in shared memory (over Q and the K/V ring, idle by
-// then) and bulk-copies each owner's rows into that owner's merge buffer.  A row is kMrgPitch floats:
+constexpr uint32_t kKVBytes = kStages * 2 * kTileBytes;  // 160 KB
+// Merge: once every CTA of the cluster has left its main loop (cluster barrier), Q and the K/V ring
+// are dead and their shared memory is reused: each CTA stages its partial rows at kOffStage and
+// bulk-copies each owner's rows into that owner's merge area at kOffMrg.  A row is kMrgPitch floats:
 // 128 accumulator columns, then the row's running maximum and sum.
 constexpr int kMrgRows = kBM + kMaxSplits;          // rows_per * n_splits <= n_valid + n_splits - 1
 constexpr int kMrgPitch = kD + 4;                   // 528-byte rows: 16-byte accesses of 32 lanes hit all banks evenly
 constexpr uint32_t kMrgRowBytes = kMrgPitch * 4;
-constexpr uint32_t kOffStage = kOffQ;               // [row][kMrgPitch] staging of this CTA's partial rows
-constexpr uint32_t kOffMrg = kOffKV + kKVBytes;
+constexpr uint32_t kOffStage = 0;                   // [row][kMrgPitch] staging of this CTA's partial rows
+constexpr uint32_t kOffMrg = ((kBM * kMrgRowBytes + 1023u) / 1024u) * 1024u;
 constexpr uint32_t kMrgBytes = kMrgRows * kMrgRowBytes;
-constexpr uint32_t kSmemBytes = kOffMrg + kMrgBytes;
+constexpr uint32_t kSmemBytes = kOffKV + kKVBytes;
 constexpr uint32_t kSmemAlloc = kSmemBytes + 1024;  // room to align the base to 1 KB
-static_assert(kBM * kMrgRowBytes <= kQBytes + kKVBytes, "staging must fit over Q and the K/V ring");
+static_assert(kOffMrg + kMrgBytes <= kSmemBytes, "staging and merge areas must fit over Q and the K/V ring");
 
 // tensor memory columns (32-bit each, 128 lanes)
 constexpr uint32_t kTmemCols = 512;
@@ -118,11 +126,25 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
     uint32_t ok;
+#if EXP_HINT == 0
+    asm volatile(
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+#elif EXP_HINT == 1
+    asm volatile(
+        "{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+#else
     asm volatile(
         "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3; selp.u32 %0, 1, 0, p; }"
         : "=r"(ok)
         : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
+#endif
     if (ok) return true;
     if ((it & 255u) == 255u && *abort_flag) return false;
   }
@@ -258,11 +280,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int kvh = blockIdx.y % p.Hkv, mtile = blockIdx.y / p.Hkv, b = blockIdx.z;
   const int G = p.G;
 
+#ifndef EXP_NOPF
   if (tid == 0) {
     prefetch_tmap(&tm_q);
     prefetch_tmap(&tm_k);
     prefetch_tmap(&tm_v);
   }
+#endif
   const int node_base = p.node_off[b];
   const int T_real = p.node_off[b + 1] - node_base;
   const int L_raw = p.prefix_len[b];
@@ -321,7 +345,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         tma_load_4d(smem_base + kOffQ, &tm_q, bar(kBarQ), 0, 0, kvh, node0);
         tma_load_4d(smem_base + kOffQ + kQBytes / 2, &tm_q, bar(kBarQ), 64, 0, kvh, node0);
       }
-      const int pre = min(n_my, kStages);
+      const int pre = min(n_my, kPrefetch);
       for (int j = 0; j < pre; ++j) {
         const int k0 = (t_begin + j) * kBN;
         const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
@@ -355,15 +379,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   tc_fence_after();
   const uint32_t tmem_base = s_tmem_base;
   FALCON_TRACE(tid == 0, 4);
-  // Cluster phase 1: "my merge barrier exists".  Arrive now, wait just before the first remote copy.
-  if (n_splits > 1) cluster_arrive();
 
   if (warp == kWarpProducer) {
     // ================================ TMA producer (ring refills) ================================
     if (lane == 0) {
-      for (int j = kStages; j < n_my; ++j) {
+      for (int j = kPrefetch; j < n_my; ++j) {
         const int st = j % kStages, u = j / kStages;
-        if (!mbar_wait(bar(kBarKVEmpty + st), (u - 1) & 1, abort_flag)) break;
+        // the next tile is requested when the oldest outstanding one has landed (and its stage is free)
+        const int jl = j - kPrefetch;
+        if (!mbar_wait(bar(kBarVFull + jl % kStages), (jl / kStages) & 1, abort_flag)) break;
+        if (u >= 1 && !mbar_wait(bar(kBarKVEmpty + st), (u - 1) & 1, abort_flag)) break;
         const int k0 = (t_begin + j) * kBN;
         const uint32_t kdst = smem_base + kOffKV + st * 2 * kTileBytes;
         const uint32_t vdst = kdst + kTileBytes;
@@ -526,6 +551,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           }
         }
         const float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale;  // -inf stays -inf
+        FALCON_TRACE(tid == 0 && j < 6 && tmax > -3e38f, 83 + 4 * j);
         if (m_used == -INFINITY) {
           m_used = tmax;  // nothing accumulated yet for this row (O and l are zero)
         } else if (tmax > m_used + kRescaleThreshold) {
@@ -554,10 +580,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         for (int c = 0; c < 32; ++c) pk[c] = 0u;
       }
 
-      FALCON_TRACE(tid == 0 && j < 6, 42 + 4 * j);
+      FALCON_TRACE(tid == 0 && j < 6 && l_sum >= 0.f, 42 + 4 * j);
       // P buffer free again?  (P.V of tile j-2 finished)
       if (u2 >= 1 && !mbar_wait_warp(bar(kBarPEmpty + sb), (u2 - 1) & 1, abort_flag)) break;
 
+      FALCON_TRACE(tid == 0 && j < 6, 80 + 4 * j);
       // rare: the row maximum jumped; rescale the accumulator before this tile is added
       if (warp_valid && __any_sync(0xffffffffu, need_rescale) && j > 0) {
         if (!mbar_wait_warp(bar(kBarPEmpty + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag)) break;
@@ -575,7 +602,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
       if (warp_valid) {
         FALCON_TMEM_ST32(tmem_lane + kTmemP + sb * 32, pk);
+        FALCON_TRACE(tid == 0 && j < 6, 81 + 4 * j);
         tmem_wait_st();
+        FALCON_TRACE(tid == 0 && j < 6, 82 + 4 * j);
       }
       tc_fence_before();
       __syncwarp();
@@ -612,7 +641,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
       }
     } else {
-      // the K/V ring is idle now (all of this CTA's MMAs have finished): stage row -> [row][kMrgPitch]
+      // Q and the K/V ring are idle now (all of this CTA's MMAs have finished): stage row -> [row][kMrgPitch]
       float* stage = reinterpret_cast<float*>(smem_gen + kOffStage) + row * kMrgPitch;
       if (have) {
 #pragma unroll 1
@@ -641,7 +670,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   FALCON_TRACE(tid == 0, 72);
   if (s_abort && tid == 0) dev_status_or(p.status, b, FALCON_DEV_TIMEOUT);
   if (n_splits > 1) {
-    cluster_wait();  // phase 1 done: every peer's merge barrier is initialised
+    // Cluster phase 1: every CTA has left its main loop and staged its rows, so the merge areas
+    // (which overlay Q and the K/V ring) may be written by peers.
+    cluster_arrive();
+    cluster_wait();
     FALCON_TRACE(tid == 0, 73);
     if (warp == kWarpProducer && lane == 0) {
       // one bulk copy per owner: its rows of this split, contiguous in the staging area
