@@ -85,12 +85,10 @@ constexpr uint32_t kTmemP = 256;    // 2 x 32 columns: bf16 pairs
 
 enum {
   kBarQ = 0,                         // the Q tile has landed in shared memory
-  kBarKFull = 1,                     // [kStages]
-  kBarVFull = kBarKFull + kStages,   // [kStages]
-  kBarKVEmpty = kBarVFull + kStages, // [kStages]
+  kBarKVFull = 1,                    // [kStages] K and V tile of the stage have landed
+  kBarKVEmpty = kBarKVFull + kStages, // [kStages]
   kBarSFull = kBarKVEmpty + kStages, // [2]
-  kBarSEmpty = kBarSFull + 2,        // [2]
-  kBarPFull = kBarSEmpty + 2,        // [2]
+  kBarPFull = kBarSFull + 2,         // [2]
   kBarPEmpty = kBarPFull + 2,        // [2]  also "P.V of tile j finished"
   kBarODone = kBarPEmpty + 2,
   kBarMrg = kBarODone + 1,           // all partial rows this CTA owns have arrived
@@ -318,13 +316,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       s_abort = 0;
       mbar_init(bar(kBarQ), 1);
       for (int s = 0; s < kStages; ++s) {
-        mbar_init(bar(kBarKFull + s), 1);
-        mbar_init(bar(kBarVFull + s), 1);
+        mbar_init(bar(kBarKVFull + s), 1);
         mbar_init(bar(kBarKVEmpty + s), 1);
       }
       for (int s = 0; s < 2; ++s) {
         mbar_init(bar(kBarSFull + s), 1);
-        mbar_init(bar(kBarSEmpty + s), n_sm_warps);
         mbar_init(bar(kBarPFull + s), n_sm_warps);
         mbar_init(bar(kBarPEmpty + s), 1);
       }
@@ -350,12 +346,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int k0 = (t_begin + j) * kBN;
         const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
         const uint32_t vdst = kdst + kTileBytes;
-        mbar_expect_tx(bar(kBarKFull + j), kTileBytes);
-        tma_load_4d(kdst, &tm_k, bar(kBarKFull + j), 0, k0, kvh, b);
-        tma_load_4d(kdst + kHalfTile, &tm_k, bar(kBarKFull + j), 64, k0, kvh, b);
-        mbar_expect_tx(bar(kBarVFull + j), kTileBytes);
-        tma_load_4d(vdst, &tm_v, bar(kBarVFull + j), 0, k0, kvh, b);
-        tma_load_4d(vdst + kHalfTile, &tm_v, bar(kBarVFull + j), 64, k0, kvh, b);
+        mbar_expect_tx(bar(kBarKVFull + j), 2 * kTileBytes);
+        tma_load_4d(kdst, &tm_k, bar(kBarKVFull + j), 0, k0, kvh, b);
+        tma_load_4d(kdst + kHalfTile, &tm_k, bar(kBarKVFull + j), 64, k0, kvh, b);
+        tma_load_4d(vdst, &tm_v, bar(kBarKVFull + j), 0, k0, kvh, b);
+        tma_load_4d(vdst + kHalfTile, &tm_v, bar(kBarKVFull + j), 64, k0, kvh, b);
       }
       FALCON_TRACE(true, 2);
       if (split == 0 && mtile == 0 && kvh == 0 && (L + T > p.s_cap || T_real > FALCON_T_MAX))
@@ -387,17 +382,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int st = j % kStages, u = j / kStages;
         // the next tile is requested when the oldest outstanding one has landed (and its stage is free)
         const int jl = j - kPrefetch;
-        if (!mbar_wait(bar(kBarVFull + jl % kStages), (jl / kStages) & 1, abort_flag)) break;
+        if (!mbar_wait(bar(kBarKVFull + jl % kStages), (jl / kStages) & 1, abort_flag)) break;
         if (u >= 1 && !mbar_wait(bar(kBarKVEmpty + st), (u - 1) & 1, abort_flag)) break;
         const int k0 = (t_begin + j) * kBN;
         const uint32_t kdst = smem_base + kOffKV + st * 2 * kTileBytes;
         const uint32_t vdst = kdst + kTileBytes;
-        mbar_expect_tx(bar(kBarKFull + st), kTileBytes);
-        tma_load_4d(kdst, &tm_k, bar(kBarKFull + st), 0, k0, kvh, b);
-        tma_load_4d(kdst + kHalfTile, &tm_k, bar(kBarKFull + st), 64, k0, kvh, b);
-        mbar_expect_tx(bar(kBarVFull + st), kTileBytes);
-        tma_load_4d(vdst, &tm_v, bar(kBarVFull + st), 0, k0, kvh, b);
-        tma_load_4d(vdst + kHalfTile, &tm_v, bar(kBarVFull + st), 64, k0, kvh, b);
+        mbar_expect_tx(bar(kBarKVFull + st), 2 * kTileBytes);
+        tma_load_4d(kdst, &tm_k, bar(kBarKVFull + st), 0, k0, kvh, b);
+        tma_load_4d(kdst + kHalfTile, &tm_k, bar(kBarKVFull + st), 64, k0, kvh, b);
+        tma_load_4d(vdst, &tm_v, bar(kBarKVFull + st), 0, k0, kvh, b);
+        tma_load_4d(vdst + kHalfTile, &tm_v, bar(kBarKVFull + st), 64, k0, kvh, b);
       }
     }
   } else if (warp == kWarpMma) {
@@ -411,7 +405,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       FALCON_TRACE(elected, 5);
       auto issue_pv = [&](int t) -> bool {
         const int st = t % kStages, pb = t & 1;
-        if (!mbar_wait_warp(bar(kBarVFull + st), (t / kStages) & 1, abort_flag)) return false;
+        FALCON_TRACE(elected && t < 6, 113 + (t - 0));
         if (!mbar_wait_warp(bar(kBarPFull + pb), (t >> 1) & 1, abort_flag)) return false;
         FALCON_TRACE(elected && t < 6, 12 + 4 * t);
         tc_fence_after();
@@ -433,8 +427,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       };
       for (int j = 0; ok && j < n_my; ++j) {
         const int st = j % kStages, sb = j & 1;
-        if (!mbar_wait_warp(bar(kBarKFull + st), (j / kStages) & 1, abort_flag)) { ok = false; break; }
-        if (j >= 2 && !mbar_wait_warp(bar(kBarSEmpty + sb), ((j >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+        // S buffer sb held the scores of tile j-2; the softmax warps read them before they wrote
+        // P(j-2), and P(j-2) was waited for before P.V of tile j-2 was issued: it is free.
+        if (!mbar_wait_warp(bar(kBarKVFull + st), (j / kStages) & 1, abort_flag)) { ok = false; break; }
         FALCON_TRACE(elected && j < 6, 10 + 4 * j);
         tc_fence_after();
         const uint32_t kbase = smem_base + kOffKV + st * 2 * kTileBytes;
@@ -496,14 +491,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         FALCON_TMEM_LD32(tmem_lane + kTmemS + sb * kBN + 32, (sr + 32));
         tmem_wait_ld();
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(kBarSEmpty + sb));
       FALCON_TRACE(tid == 0 && j < 6, 41 + 4 * j);
 
       // the sequence's last tile: rows of V past the last key may hold anything (0 x NaN = NaN in the MMA)
       if (k0 + kBN > S_valid) {
-        if (!mbar_wait_warp(bar(kBarVFull + st), (j / kStages) & 1, abort_flag)) break;
+        if (!mbar_wait_warp(bar(kBarKVFull + st), (j / kStages) & 1, abort_flag)) break;
         const int nv = S_valid - k0;  // 1..63 rows are real
         unsigned char* vtile = smem_gen + kOffKV + st * 2 * kTileBytes + kTileBytes;
         const int chunks = (kBN - nv) * 8;
@@ -581,8 +573,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
 
       FALCON_TRACE(tid == 0 && j < 6 && l_sum >= 0.f, 42 + 4 * j);
-      // P buffer free again?  (P.V of tile j-2 finished)
-      if (u2 >= 1 && !mbar_wait_warp(bar(kBarPEmpty + sb), (u2 - 1) & 1, abort_flag)) break;
+      // P buffer sb is free: the commit behind S(j) covers every MMA issued before it, and P.V of
+      // tile j-2 was issued before Q.K^T of tile j.
 
       FALCON_TRACE(tid == 0 && j < 6, 80 + 4 * j);
       // rare: the row maximum jumped; rescale the accumulator before this tile is added
@@ -610,6 +602,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(kBarPFull + sb));
       FALCON_TRACE(tid == 0 && j < 6, 43 + 4 * j);
+      FALCON_TRACE(tid == 32 && j < 6, 107 + (j - 0));
     }
 
     // ---- this split's partial rows: straight to global (one split) or staged for the merge ----
