@@ -193,8 +193,10 @@ def run_falcon(args):
 
     node_off, parent, token, prefix = i32(tb.node_off), i32(tb.parent), i32(tb.token), i32(tb.prefix_len)
     status = torch.zeros(B, dtype=torch.int32, device=dev)
+    host_prefix = np.ascontiguousarray(tb.prefix_len, dtype=np.int32)   # the caller knows these: no device round trip
+    host_node_off = np.ascontiguousarray(tb.node_off, dtype=np.int32)
     tree = binding.tree_desc(B, N, tb.max_tree, int(tb.prefix_len.max()), node_off, parent, prefix, token=token,
-                             status=status)
+                             prefix_len_host=host_prefix, node_off_host=host_node_off, status=status)
 
     # all layers' caches in one allocation [NL, 2, B, Hkv, s_cap, D]; q and out [NL, N, Hq, D]
     cache = torch.empty((NL, 2, B, Hkv, s_cap, D), dtype=torch.bfloat16, device=dev)

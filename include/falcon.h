@@ -85,7 +85,9 @@ typedef struct {
   const int32_t* parent;          /* [N] local parent index, -1 at each local node 0    */
   const int32_t* token;           /* [N] drafted token ids (used by accept only)        */
   const int32_t* prefix_len;      /* [B] rows of the cache that hold the prefix         */
-  const int32_t* prefix_len_host; /* optional HOST copy of prefix_len (scheduling hint) */
+  const int32_t* prefix_len_host; /* optional HOST copy of prefix_len                   */
+  const int32_t* node_off_host;   /* optional HOST copy of node_off.  With both host copies (they must
+                                     equal the device arrays) small batches skip a device round trip */
   int32_t* status;                /* optional [B] device status words (FALCON_DEV_*)    */
 } falcon_tree_desc;
 

@@ -31,7 +31,7 @@ class TreeDesc(C.Structure):
     _fields_ = [("batch", C.c_int32), ("total_nodes", C.c_int32), ("max_tree", C.c_int32),
                 ("max_prefix_len", C.c_int32), ("node_off", C.c_void_p), ("parent", C.c_void_p),
                 ("token", C.c_void_p), ("prefix_len", C.c_void_p), ("prefix_len_host", C.c_void_p),
-                ("status", C.c_void_p)]
+                ("node_off_host", C.c_void_p), ("status", C.c_void_p)]
 
 
 class AttnArgs(C.Structure):
@@ -131,9 +131,12 @@ def _stream(stream) -> Optional[int]:
 
 
 def tree_desc(batch, total_nodes, max_tree, max_prefix_len, node_off, parent, prefix_len, token=None,
-              prefix_len_host=None, status=None) -> TreeDesc:
+              prefix_len_host=None, node_off_host=None, status=None) -> TreeDesc:
+    """prefix_len_host / node_off_host: optional host int32 numpy arrays (kept alive by the caller)."""
+    def host(a):
+        return None if a is None else a.ctypes.data
     return TreeDesc(batch, total_nodes, max_tree, max_prefix_len, _ptr(node_off), _ptr(parent), _ptr(token),
-                    _ptr(prefix_len), prefix_len_host, _ptr(status))
+                    _ptr(prefix_len), host(prefix_len_host), host(node_off_host), _ptr(status))
 
 
 class Context:

@@ -42,19 +42,17 @@ constexpr int kD = 128;
 constexpr int kBM = 128;          // query rows per CTA (TMEM lanes)
 constexpr int kBN = 64;           // keys per tile
 constexpr int kStages = 5;
-#ifndef EXP_PREFETCH
-#define EXP_PREFETCH 5
-#endif
-constexpr int kPrefetch = EXP_PREFETCH;  // tiles requested ahead of the consumer (<= kStages)
+// Tiles requested ahead of the consumer.  Small on purpose: everything a CTA asks for at once
+// arrives together (the memory system serves the whole GPU's requests fairly), so a deep burst only
+// delays the first tile; the ring still lets the producer run ahead once tiles are consumed.
+constexpr int kPrefetch = 2;
 constexpr int kTcThreads = 256;    // warps 0-3 softmax (TMEM quadrant = warp), 4-5 idle, 6 producer, 7 MMA
 constexpr int kWarpProducer = 6;
 constexpr int kWarpMma = 7;
 constexpr int kMaxSplits = 8;
+constexpr int kHostSeqs = 8;
 constexpr uint32_t kSpinLimit = 1u << 18;
-#ifndef EXP_HINT
-#define EXP_HINT 2000
-#endif
-constexpr uint32_t kSuspendHintNs = EXP_HINT;  // a waiting thread may sleep this long per try (it wakes when the phase completes)
+constexpr uint32_t kSuspendHintNs = 2000;  // a waiting thread may sleep this long per try (it wakes when the phase completes)
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 constexpr uint32_t kTileBytes = kBN * kD * 2;      // 16 KB: two 64-column halves of 8 KB
@@ -97,6 +95,7 @@ enum {
 
 struct TcParams {
   int32_t Hq, Hkv, G, s_cap, total_nodes;
+  uint32_t q_half_bytes;  // bytes of one 64-column half of the Q tile as loaded (rows of the box x 128)
   float scale_log2;
   const int32_t* node_off;
   const int32_t* parent;
@@ -105,6 +104,11 @@ struct TcParams {
   const uint64_t* tree_mask;
   const __nv_bfloat16* q;
   __nv_bfloat16* out;
+  // Per-sequence scalars from the caller's host copies (batches of up to kHostSeqs sequences):
+  // with them the first loads do not have to wait for a round trip to global memory.
+  int32_t have_host;
+  int32_t h_node_off[kHostSeqs + 1];
+  int32_t h_prefix[kHostSeqs];
 };
 
 // ------------------------------------------------------------------------------------ PTX helpers
@@ -124,25 +128,11 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
     uint32_t ok;
-#if EXP_HINT == 0
-    asm volatile(
-        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-#elif EXP_HINT == 1
-    asm volatile(
-        "{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-#else
     asm volatile(
         "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3; selp.u32 %0, 1, 0, p; }"
         : "=r"(ok)
         : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
-#endif
     if (ok) return true;
     if ((it & 255u) == 255u && *abort_flag) return false;
   }
@@ -155,12 +145,17 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
   return __all_sync(0xffffffffu, ok);
 }
 
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
-                                            int c3) {
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3, int c4) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], "
+      "[%2];" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
       : "memory");
+}
+// One K or V tile: 64 keys x (2 halves of 64 head-dim columns), landing as two 128-byte-swizzled half tiles.
+__device__ __forceinline__ void load_kv_tile(uint32_t dst, const CUtensorMap* map, uint32_t bar, int k0, int kvh, int b) {
+  tma_load_5d(dst, map, bar, 0, k0, 0, kvh, b);
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -278,16 +273,21 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int kvh = blockIdx.y % p.Hkv, mtile = blockIdx.y / p.Hkv, b = blockIdx.z;
   const int G = p.G;
 
-#ifndef EXP_NOPF
   if (tid == 0) {
     prefetch_tmap(&tm_q);
     prefetch_tmap(&tm_k);
     prefetch_tmap(&tm_v);
   }
-#endif
-  const int node_base = p.node_off[b];
-  const int T_real = p.node_off[b + 1] - node_base;
-  const int L_raw = p.prefix_len[b];
+  int node_base, T_real, L_raw;
+  if (p.have_host) {
+    node_base = p.h_node_off[b];
+    T_real = p.h_node_off[b + 1] - node_base;
+    L_raw = p.h_prefix[b];
+  } else {
+    node_base = p.node_off[b];
+    T_real = p.node_off[b + 1] - node_base;
+    L_raw = p.prefix_len[b];
+  }
   const int T = min(T_real, FALCON_T_MAX);
   const int rows_total = T * G;
   if (mtile * kBM >= rows_total) return;  // same decision in every CTA of the cluster
@@ -295,10 +295,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int L = max(L_raw, 0);
   const int Lc = min(L, p.s_cap);
   const int S_valid = min(L + T, p.s_cap);  // keys that exist below the cache capacity
+  // Whole tiles per split, as even as they go (an iteration costs about the same whatever part of
+  // its 64 keys is real, so fewer iterations beat equal key counts).
   const int n_tiles = (S_valid + kBN - 1) / kBN;
-  const int t_begin = (split * n_tiles) / n_splits;
-  const int t_end = ((split + 1) * n_tiles) / n_splits;
-  const int n_my = t_end - t_begin;
+  const int key_begin = min(S_valid, ((split * n_tiles) / n_splits) * kBN);
+  const int key_end = min(S_valid, (((split + 1) * n_tiles) / n_splits) * kBN);
+  const int n_my = (key_end - key_begin + kBN - 1) / kBN;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -310,70 +312,63 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int rows_per = (n_valid + n_splits - 1) / n_splits;
 
   const int n_sm_warps = (n_valid + 31) >> 5;  // softmax warps that own at least one query row
-  if (warp == kWarpProducer) {
-    if (lane == 0) {
-      FALCON_TRACE(true, 1);
-      s_abort = 0;
-      mbar_init(bar(kBarQ), 1);
-      for (int s = 0; s < kStages; ++s) {
-        mbar_init(bar(kBarKVFull + s), 1);
-        mbar_init(bar(kBarKVEmpty + s), 1);
-      }
-      for (int s = 0; s < 2; ++s) {
-        mbar_init(bar(kBarSFull + s), 1);
-        mbar_init(bar(kBarPFull + s), n_sm_warps);
-        mbar_init(bar(kBarPEmpty + s), 1);
-      }
-      mbar_init(bar(kBarODone), 1);
-      mbar_init(bar(kBarMrg), 1);
-      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-      if (n_splits > 1) {
-        // this CTA will receive rows_mine rows from every split (its own included)
-        const int r0 = split * rows_per;
-        const int mine = max(0, min(n_valid, r0 + rows_per) - r0);
-        mbar_expect_tx(bar(kBarMrg), static_cast<uint32_t>(n_splits * mine) * kMrgRowBytes);
-      }
-      // first loads right away (they need nothing but the barriers this thread just made), Q in front
-      // so that it is not queued behind the K/V tiles
-      if (n_my > 0) {
-        const int node0 = node_base + mtile * (kBM / G);
-        mbar_expect_tx(bar(kBarQ), kQBytes);
-        tma_load_4d(smem_base + kOffQ, &tm_q, bar(kBarQ), 0, 0, kvh, node0);
-        tma_load_4d(smem_base + kOffQ + kQBytes / 2, &tm_q, bar(kBarQ), 64, 0, kvh, node0);
-      }
-      const int pre = min(n_my, kPrefetch);
-      for (int j = 0; j < pre; ++j) {
-        const int k0 = (t_begin + j) * kBN;
-        const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
-        const uint32_t vdst = kdst + kTileBytes;
-        mbar_expect_tx(bar(kBarKVFull + j), 2 * kTileBytes);
-        tma_load_4d(kdst, &tm_k, bar(kBarKVFull + j), 0, k0, kvh, b);
-        tma_load_4d(kdst + kHalfTile, &tm_k, bar(kBarKVFull + j), 64, k0, kvh, b);
-        tma_load_4d(vdst, &tm_v, bar(kBarKVFull + j), 0, k0, kvh, b);
-        tma_load_4d(vdst + kHalfTile, &tm_v, bar(kBarKVFull + j), 64, k0, kvh, b);
-      }
-      FALCON_TRACE(true, 2);
-      if (split == 0 && mtile == 0 && kvh == 0 && (L + T > p.s_cap || T_real > FALCON_T_MAX))
-        dev_status_or(p.status, b, FALCON_DEV_CAPACITY);
-    }
-    __syncwarp();
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
-                 "r"(kTmemCols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-
   const int q4 = warp & 3;
   const int row = q4 * 32 + lane;
   const bool is_sm = warp < 4;
   const bool valid = is_sm && row < n_valid;
   const bool warp_valid = is_sm && q4 * 32 < n_valid;
 
+  if (warp == kWarpProducer) {
+    FALCON_TRACE(lane == 0, 1);
+    if (lane == 0) s_abort = 0;
+    if (lane < kNumBars) {  // barrier i is initialised by lane i
+      const bool per_warp = lane == kBarPFull || lane == kBarPFull + 1;
+      mbar_init(bar(lane), per_warp ? n_sm_warps : 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  } else if (warp == kWarpMma) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = s_tmem_base;
   FALCON_TRACE(tid == 0, 4);
+
+  // First loads, issued by several warps at once (a TMA instruction costs its issuing thread about
+  // a hundred cycles): the producer takes the Q tile, in front so that it is not queued behind K/V,
+  // and the last stage; lane 0 of warps 0-3 takes stages 0-3.
+  {
+    const int pre = min(n_my, kPrefetch);
+    if (lane == 0 && (is_sm || warp == kWarpProducer)) {
+      if (warp == kWarpProducer) {
+        if (n_splits > 1) {
+          // this CTA will receive rows_mine rows from every split (its own included)
+          const int r0 = split * rows_per;
+          const int mine = max(0, min(n_valid, r0 + rows_per) - r0);
+          mbar_expect_tx(bar(kBarMrg), static_cast<uint32_t>(n_splits * mine) * kMrgRowBytes);
+        }
+        if (n_my > 0) {
+          mbar_expect_tx(bar(kBarQ), 2 * p.q_half_bytes);
+          tma_load_5d(smem_base + kOffQ, &tm_q, bar(kBarQ), 0, 0, kvh, node_base + mtile * (kBM / G), 0);
+        }
+        if (split == 0 && mtile == 0 && kvh == 0 && (L + T > p.s_cap || T_real > FALCON_T_MAX))
+          dev_status_or(p.status, b, FALCON_DEV_CAPACITY);
+      }
+      // warps 0-3: one stage each; the producer: whatever is left
+      for (int j = is_sm ? warp : 4; j < pre; j += is_sm ? kStages : 1) {
+        const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
+        mbar_expect_tx(bar(kBarKVFull + j), 2 * kTileBytes);
+        load_kv_tile(kdst, &tm_k, bar(kBarKVFull + j), key_begin + j * kBN, kvh, b);
+        load_kv_tile(kdst + kTileBytes, &tm_v, bar(kBarKVFull + j), key_begin + j * kBN, kvh, b);
+      }
+    }
+    __syncwarp();
+    FALCON_TRACE(warp == kWarpProducer && lane == 0, 2);
+  }
 
   if (warp == kWarpProducer) {
     // ================================ TMA producer (ring refills) ================================
@@ -384,14 +379,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int jl = j - kPrefetch;
         if (!mbar_wait(bar(kBarKVFull + jl % kStages), (jl / kStages) & 1, abort_flag)) break;
         if (u >= 1 && !mbar_wait(bar(kBarKVEmpty + st), (u - 1) & 1, abort_flag)) break;
-        const int k0 = (t_begin + j) * kBN;
+        const int k0 = key_begin + j * kBN;
         const uint32_t kdst = smem_base + kOffKV + st * 2 * kTileBytes;
         const uint32_t vdst = kdst + kTileBytes;
         mbar_expect_tx(bar(kBarKVFull + st), 2 * kTileBytes);
-        tma_load_4d(kdst, &tm_k, bar(kBarKVFull + st), 0, k0, kvh, b);
-        tma_load_4d(kdst + kHalfTile, &tm_k, bar(kBarKVFull + st), 64, k0, kvh, b);
-        tma_load_4d(vdst, &tm_v, bar(kBarKVFull + st), 0, k0, kvh, b);
-        tma_load_4d(vdst + kHalfTile, &tm_v, bar(kBarKVFull + st), 64, k0, kvh, b);
+        load_kv_tile(kdst, &tm_k, bar(kBarKVFull + st), k0, kvh, b);
+        load_kv_tile(vdst, &tm_v, bar(kBarKVFull + st), k0, kvh, b);
       }
     }
   } else if (warp == kWarpMma) {
@@ -437,7 +430,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
           for (int kk = 0; kk < kD / 16; ++kk) {
             // Q and K tiles: K-major, 16 head-dim columns = 32 bytes inside the 128-byte swizzle row
-            const uint64_t ad = smem_desc(smem_base + kOffQ + (kk >> 2) * (kQBytes / 2) + (kk & 3) * 32, 16, 1024);
+            const uint64_t ad = smem_desc(smem_base + kOffQ + (kk >> 2) * p.q_half_bytes + (kk & 3) * 32, 16, 1024);
             const uint64_t bd = smem_desc(kbase + (kk >> 2) * kHalfTile + (kk & 3) * 32, 16, 1024);
             umma_bf16_ss(tmem_base + kTmemS + sb * kBN, ad, bd, kIdescQK, kk > 0 ? 1u : 0u);
           }
@@ -481,7 +474,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
     for (int j = 0; j < n_my; ++j) {
       const int sb = j & 1, u2 = j >> 1, st = j % kStages;
-      const int k0 = (t_begin + j) * kBN;
+      const int k0 = key_begin + j * kBN;
       if (!mbar_wait_warp(bar(kBarSFull + sb), u2 & 1, abort_flag)) break;
       FALCON_TRACE(tid == 0 && j < 6, 40 + 4 * j);
       tc_fence_after();
@@ -514,7 +507,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         // guaranteed by the launcher, so the maximum can be taken on the raw scores)
         float s[64];
         float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-        if (k0 + kBN <= Lc) {
+        if (k0 + kBN <= min(Lc, key_end)) {
 #pragma unroll
           for (int c = 0; c < 64; c += 4) {
             s[c] = __uint_as_float(sr[c]);
@@ -527,7 +520,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             mx3 = fmaxf(mx3, s[c + 3]);
           }
         } else {
-          const uint64_t vis = window64(anc_lo, anc_hi, k0 - Lc);
+          uint64_t vis = window64(anc_lo, anc_hi, k0 - Lc);
+          if (key_end - k0 < kBN) vis &= (1ull << (key_end - k0)) - 1ull;  // keys of the next split
           const uint32_t vlo = static_cast<uint32_t>(vis), vhi = static_cast<uint32_t>(vis >> 32);
 #pragma unroll
           for (int c = 0; c < 64; c += 4) {
@@ -730,7 +724,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     cluster_wait();
     FALCON_TRACE(tid == 0, 76);
   }
-  if (warp == kWarpProducer) {
+  if (warp == kWarpMma) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
@@ -755,9 +749,9 @@ EncodeFn get_encode() {
 
 struct TmapEntry {
   const void* base;
-  uint64_t dims[4];
-  uint64_t strides[3];
-  uint32_t box[4];
+  uint64_t dims[5];
+  uint64_t strides[4];
+  uint32_t box[5];
   CUtensorMap map;
 };
 
@@ -765,16 +759,16 @@ struct TmapCache {
   std::vector<TmapEntry> entries;
 };
 
-// 4-D bf16 tensor map with 128-byte swizzle; cached per (base, shape, strides, box).
-const CUtensorMap* get_tmap(falcon_ctx* ctx, const void* base, const uint64_t dims[4], const uint64_t strides[3],
-                            const uint32_t box[4]) {
+// 5-D bf16 tensor map with 128-byte swizzle; cached per (base, shape, strides, box).
+const CUtensorMap* get_tmap(falcon_ctx* ctx, const void* base, const uint64_t dims[5], const uint64_t strides[4],
+                            const uint32_t box[5]) {
   if (!ctx->tmap_cache) ctx->tmap_cache = new TmapCache();
   TmapCache* cache = static_cast<TmapCache*>(ctx->tmap_cache);
   for (TmapEntry& e : cache->entries) {
     if (e.base != base) continue;
     bool same = true;
-    for (int i = 0; i < 4; ++i) same = same && e.dims[i] == dims[i] && e.box[i] == box[i];
-    for (int i = 0; i < 3; ++i) same = same && e.strides[i] == strides[i];
+    for (int i = 0; i < 5; ++i) same = same && e.dims[i] == dims[i] && e.box[i] == box[i];
+    for (int i = 0; i < 4; ++i) same = same && e.strides[i] == strides[i];
     if (same) return &e.map;
   }
   EncodeFn enc = get_encode();
@@ -782,11 +776,11 @@ const CUtensorMap* get_tmap(falcon_ctx* ctx, const void* base, const uint64_t di
   if (cache->entries.size() >= 4096) cache->entries.clear();
   TmapEntry e;
   e.base = base;
-  for (int i = 0; i < 4; ++i) { e.dims[i] = dims[i]; e.box[i] = box[i]; }
-  for (int i = 0; i < 3; ++i) e.strides[i] = strides[i];
-  const cuuint32_t elem[4] = {1, 1, 1, 1};
+  for (int i = 0; i < 5; ++i) { e.dims[i] = dims[i]; e.box[i] = box[i]; }
+  for (int i = 0; i < 4; ++i) e.strides[i] = strides[i];
+  const cuuint32_t elem[5] = {1, 1, 1, 1, 1};
   alignas(64) CUtensorMap m;
-  CUresult r = enc(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, elem,
+  CUresult r = enc(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, elem,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return nullptr;
@@ -855,20 +849,27 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
     attr_set = true;
   }
 
-  // tensor maps of the K and V caches: [D, s_cap, Hkv, B], box 64 x 64 (one half tile)
-  uint64_t kv_dims[4] = {static_cast<uint64_t>(kD), static_cast<uint64_t>(a.s_cap), static_cast<uint64_t>(Hkv),
-                         static_cast<uint64_t>(B)};
-  uint64_t kv_strides[3] = {static_cast<uint64_t>(a.kv_stride_s) * 2, static_cast<uint64_t>(a.kv_stride_h) * 2,
+  // Tensor maps.  The head dimension is split into (64 columns, 2 halves) so that one box covers both
+  // 128-byte-swizzled half tiles.  K/V cache: [64, s_cap, 2, Hkv, B], box 64 x 64 keys x 2.
+  uint64_t kv_dims[5] = {64, static_cast<uint64_t>(a.s_cap), 2, static_cast<uint64_t>(Hkv), static_cast<uint64_t>(B)};
+  uint64_t kv_strides[4] = {static_cast<uint64_t>(a.kv_stride_s) * 2, 128, static_cast<uint64_t>(a.kv_stride_h) * 2,
                             static_cast<uint64_t>(a.kv_stride_b) * 2};
-  if (Hkv == 1 && kv_strides[1] == 0) kv_strides[1] = kv_strides[0] * a.s_cap;  // a size-1 dimension never strides
-  if (B == 1 && kv_strides[2] == 0) kv_strides[2] = kv_strides[1] * Hkv;
-  const uint32_t kv_box[4] = {64, static_cast<uint32_t>(kBN), 1, 1};
-  // q [D, G, Hkv, N]: one box is the 128 query rows (128/G nodes x G heads) of a KV head, half of D
+  if (Hkv == 1 && kv_strides[2] == 0) kv_strides[2] = kv_strides[0] * a.s_cap;  // a size-1 dimension never strides
+  if (B == 1 && kv_strides[3] == 0) kv_strides[3] = kv_strides[2] * Hkv;
+  const uint32_t kv_box[5] = {64, static_cast<uint32_t>(kBN), 2, 1, 1};
+  // q: [64, G, Hkv, N, 2]; a box is the query rows of one KV head: q_nodes nodes x G heads (at most
+  // 128 rows, a multiple of 8 so that the second half starts on a swizzle-atom boundary)
   const uint64_t row_bytes = static_cast<uint64_t>(kD) * 2;
-  uint64_t q_dims[4] = {static_cast<uint64_t>(kD), static_cast<uint64_t>(G), static_cast<uint64_t>(Hkv),
-                        static_cast<uint64_t>(a.tree.total_nodes)};
-  uint64_t q_strides[3] = {row_bytes, row_bytes * G, row_bytes * Hq};
-  const uint32_t q_box[4] = {64, static_cast<uint32_t>(G), 1, static_cast<uint32_t>(kBM / G)};
+  int q_nodes = kBM / G;
+  {
+    const int gran = G >= 8 ? 1 : 8 / G;
+    const int want = (a.tree.max_tree + gran - 1) / gran * gran;
+    if (want < q_nodes) q_nodes = want;
+  }
+  uint64_t q_dims[5] = {64, static_cast<uint64_t>(G), static_cast<uint64_t>(Hkv),
+                        static_cast<uint64_t>(a.tree.total_nodes), 2};
+  uint64_t q_strides[4] = {row_bytes, row_bytes * G, row_bytes * Hq, 128};
+  const uint32_t q_box[5] = {64, static_cast<uint32_t>(G), 1, static_cast<uint32_t>(q_nodes), 2};
   const CUtensorMap* tq = get_tmap(ctx, a.q, q_dims, q_strides, q_box);
   const CUtensorMap* tk = get_tmap(ctx, a.k_cache, kv_dims, kv_strides, kv_box);
   const CUtensorMap* tv = get_tmap(ctx, a.v_cache, kv_dims, kv_strides, kv_box);
@@ -890,11 +891,18 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   p.s_cap = a.s_cap;
   p.total_nodes = a.tree.total_nodes;
   p.scale_log2 = a.sm_scale * kLog2e;
+  p.q_half_bytes = static_cast<uint32_t>(q_nodes) * G * 128u;
   p.node_off = a.tree.node_off;
   p.parent = a.tree.parent;
   p.prefix_len = a.tree.prefix_len;
   p.status = a.tree.status;
   p.tree_mask = a.tree_mask;
+  p.have_host = 0;
+  if (a.tree.prefix_len_host && a.tree.node_off_host && B <= kHostSeqs) {
+    p.have_host = 1;
+    for (int i = 0; i <= B; ++i) p.h_node_off[i] = a.tree.node_off_host[i];
+    for (int i = 0; i < B; ++i) p.h_prefix[i] = a.tree.prefix_len_host[i];
+  }
   p.q = static_cast<const __nv_bfloat16*>(a.q);
   p.out = static_cast<__nv_bfloat16*>(a.out);
 

@@ -45,10 +45,15 @@ class DevTrees:
         self.status = torch.zeros(trees.batch, dtype=torch.int32, device="cuda")
         self.max_prefix_len = int(max(0, trees.prefix_len.max())) if max_prefix_len is None else max_prefix_len
 
-    def desc(self, with_status=True):
+    def desc(self, with_status=True, host_copies=False):
         t = self.host
+        self._host_keep = (np.ascontiguousarray(t.prefix_len, dtype=np.int32),
+                           np.ascontiguousarray(t.node_off, dtype=np.int32))
         return binding.tree_desc(t.batch, t.total_nodes, t.max_tree, self.max_prefix_len, self.node_off, self.parent,
-                                 self.prefix_len, token=self.token, status=self.status if with_status else None)
+                                 self.prefix_len, token=self.token,
+                                 prefix_len_host=self._host_keep[0] if host_copies else None,
+                                 node_off_host=self._host_keep[1] if host_copies else None,
+                                 status=self.status if with_status else None)
 
 
 def make_trees(sizes, prefs, rng, vocab=100, parents=None) -> synth.TreeBatch:
@@ -61,7 +66,7 @@ def make_trees(sizes, prefs, rng, vocab=100, parents=None) -> synth.TreeBatch:
 
 
 def run_attn(dt: DevTrees, Hq, Hkv, D, q, k, v, s_cap=None, scale=None, kernel=binding.ATTN_AUTO, n_splits=0,
-             k_tree=None, v_tree=None, tree_mask=None, check=True):
+             k_tree=None, v_tree=None, tree_mask=None, check=True, host_copies=False):
     """q [N,Hq,D], k/v [B,Hkv,s_cap,D] uint16 bit patterns -> (out bits [N,Hq,D], rc)."""
     scale = 1.0 / math.sqrt(D) if scale is None else scale
     qd, kd, vd = dev_bf16(q), dev_bf16(k), dev_bf16(v)
@@ -70,7 +75,7 @@ def run_attn(dt: DevTrees, Hq, Hkv, D, q, k, v, s_cap=None, scale=None, kernel=b
     vtd = dev_bf16(v_tree) if v_tree is not None else None
     md = torch.from_numpy(np.ascontiguousarray(tree_mask).view(np.int64)).cuda() if tree_mask is not None else None
     strides = tuple(int(s) for s in kd.stride()[:3])
-    a = binding.attn_args(dt.desc(), Hq, Hkv, D, scale, qd, out, kd, vd, strides,
+    a = binding.attn_args(dt.desc(host_copies=host_copies), Hq, Hkv, D, scale, qd, out, kd, vd, strides,
                           kd.shape[2] if s_cap is None else s_cap, k_tree=ktd, v_tree=vtd, tree_mask=md,
                           kernel=kernel, n_splits=n_splits)
     rc = ctx().falcon_tree_attn(a, check=check)

@@ -86,6 +86,20 @@ def test_attn_split_invariance_and_determinism(kernel):
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
+def test_attn_host_copies_of_the_scalars_change_nothing(kernel):
+    rng = np.random.default_rng(22)
+    for sizes, prefs in (([60], [1024]), ([20, 80, 33], [300, 40, 129]), ([7] * 9, [65] * 9)):   # 9 > host table size
+        tb, q, k, v = random_case(rng, sizes, prefs, 4, 2, 128, slack=2)
+        ref = oracle_attn(tb, 4, 2, 128, q, k, v)
+        dt = H.DevTrees(tb)
+        a, rc = H.run_attn(dt, 4, 2, 128, q, k, v, kernel=kernel, check=False)
+        tc_or_skip(rc)
+        b, _ = H.run_attn(dt, 4, 2, 128, q, k, v, kernel=kernel, host_copies=True)
+        np.testing.assert_array_equal(a, b)
+        H.assert_attn_close(b, ref, tb.node_off)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
 def test_attn_ragged_batch_small(kernel):
     rng = np.random.default_rng(21)
     sizes = [20, 80, 1, 47, 64, 33]
