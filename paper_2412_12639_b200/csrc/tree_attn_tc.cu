@@ -19,7 +19,7 @@
 //             warps sit on other schedulers than the first two softmax warps):
 //             per tile tcgen05.ld of the score row, tree mask from the node's ancestor bit
 //             set, online softmax with a lazily updated maximum (the accumulator is
-//             rescaled only when the row maximum grows by more than 2^8), P written back
+//             rescaled only when a weight would exceed 2^8), P written back
 //             to TMEM as packed bf16.
 // Every mbarrier wait is bounded; a wait that runs out sets FALCON_DEV_TIMEOUT in the
 // status word, and the CTA still reaches the cluster barrier and frees its TMEM.
@@ -53,7 +53,7 @@ constexpr int kMaxSplits = 8;
 constexpr int kHostSeqs = 8;
 constexpr uint32_t kSpinLimit = 1u << 18;
 constexpr uint32_t kSuspendHintNs = 2000;  // a waiting thread may sleep this long per try (it wakes when the phase completes)
-constexpr float kRescaleThreshold = 8.0f;  // log2 units
+constexpr float kRescaleLimit = 256.f;  // largest weight tolerated before the row maximum is refreshed
 
 constexpr uint32_t kTileBytes = kBN * kD * 2;      // 16 KB: two 64-column halves of 8 KB
 constexpr uint32_t kHalfTile = kBN * 128;          // 8 KB
@@ -504,9 +504,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       bool need_rescale = false;
       if (valid) {
         // scores stay raw; exp2(s * scale - m) is one FFMA + one MUFU per element (scale > 0 is
-        // guaranteed by the launcher, so the maximum can be taken on the raw scores)
+        // guaranteed by the launcher, so a maximum can be taken on the raw scores)
         float s[64];
-        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
         if (k0 + kBN <= min(Lc, key_end)) {
 #pragma unroll
           for (int c = 0; c < 64; c += 4) {
@@ -514,10 +513,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             s[c + 1] = __uint_as_float(sr[c + 1]);
             s[c + 2] = __uint_as_float(sr[c + 2]);
             s[c + 3] = __uint_as_float(sr[c + 3]);
-            mx0 = fmaxf(mx0, s[c]);
-            mx1 = fmaxf(mx1, s[c + 1]);
-            mx2 = fmaxf(mx2, s[c + 2]);
-            mx3 = fmaxf(mx3, s[c + 3]);
           }
         } else {
           uint64_t vis = window64(anc_lo, anc_hi, k0 - Lc);
@@ -530,36 +525,53 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             s[c + 1] = ((w >> ((c + 1) & 31)) & 1u) ? __uint_as_float(sr[c + 1]) : -INFINITY;
             s[c + 2] = ((w >> ((c + 2) & 31)) & 1u) ? __uint_as_float(sr[c + 2]) : -INFINITY;
             s[c + 3] = ((w >> ((c + 3) & 31)) & 1u) ? __uint_as_float(sr[c + 3]) : -INFINITY;
+          }
+        }
+        // One pass of exponentials against the maximum known so far.  The largest p tells whether
+        // that maximum is still good enough (p <= 2^8); only the first tile of a row, or a row whose
+        // scores jumped, needs the true maximum of this tile first.
+        float pmx0 = 0.f, pmx1 = 0.f, add0 = 0.f, add1 = 0.f, add2 = 0.f, add3 = 0.f;
+        auto exp_pass = [&](float neg_m) {
+          pmx0 = pmx1 = add0 = add1 = add2 = add3 = 0.f;
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            const float p0 = ex2(fmaf(s[2 * c], scale, neg_m)), p1 = ex2(fmaf(s[2 * c + 1], scale, neg_m));
+            const float p2 = ex2(fmaf(s[2 * c + 2], scale, neg_m)), p3 = ex2(fmaf(s[2 * c + 3], scale, neg_m));
+            add0 += p0;
+            add1 += p1;
+            add2 += p2;
+            add3 += p3;
+            pmx0 = fmaxf(pmx0, fmaxf(p0, p1));
+            pmx1 = fmaxf(pmx1, fmaxf(p2, p3));
+            const __nv_bfloat162 h0 = __floats2bfloat162_rn(p0, p1), h1 = __floats2bfloat162_rn(p2, p3);
+            pk[c] = *reinterpret_cast<const uint32_t*>(&h0);
+            pk[c + 1] = *reinterpret_cast<const uint32_t*>(&h1);
+          }
+        };
+        bool redo = (m_used == -INFINITY);
+        if (!redo) {
+          exp_pass(-m_used);
+          redo = !(fmaxf(pmx0, pmx1) <= kRescaleLimit);  // also catches an overflow to +inf
+        }
+        if (redo) {
+          float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+          for (int c = 0; c < 64; c += 4) {
             mx0 = fmaxf(mx0, s[c]);
             mx1 = fmaxf(mx1, s[c + 1]);
             mx2 = fmaxf(mx2, s[c + 2]);
             mx3 = fmaxf(mx3, s[c + 3]);
           }
-        }
-        const float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale;  // -inf stays -inf
-        FALCON_TRACE(tid == 0 && j < 6 && tmax > -3e38f, 83 + 4 * j);
-        if (m_used == -INFINITY) {
-          m_used = tmax;  // nothing accumulated yet for this row (O and l are zero)
-        } else if (tmax > m_used + kRescaleThreshold) {
-          alpha = ex2(m_used - tmax);
-          l_sum *= alpha;
+          const float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale;  // -inf stays -inf
+          if (m_used != -INFINITY) {  // what is accumulated so far moves to the new maximum
+            alpha = ex2(m_used - tmax);
+            l_sum *= alpha;
+            need_rescale = true;
+          }
           m_used = tmax;
-          need_rescale = true;
+          exp_pass(m_used == -INFINITY ? 0.f : -m_used);
         }
-        const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-        float add0 = 0.f, add1 = 0.f, add2 = 0.f, add3 = 0.f;
-#pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          const float p0 = ex2(fmaf(s[2 * c], scale, neg_m)), p1 = ex2(fmaf(s[2 * c + 1], scale, neg_m));
-          const float p2 = ex2(fmaf(s[2 * c + 2], scale, neg_m)), p3 = ex2(fmaf(s[2 * c + 3], scale, neg_m));
-          add0 += p0;
-          add1 += p1;
-          add2 += p2;
-          add3 += p3;
-          const __nv_bfloat162 h0 = __floats2bfloat162_rn(p0, p1), h1 = __floats2bfloat162_rn(p2, p3);
-          pk[c] = *reinterpret_cast<const uint32_t*>(&h0);
-          pk[c + 1] = *reinterpret_cast<const uint32_t*>(&h1);
-        }
+        FALCON_TRACE(tid == 0 && j < 6 && pmx0 >= 0.f, 83 + 4 * j);
         l_sum += (add0 + add1) + (add2 + add3);
       } else {
 #pragma unroll
