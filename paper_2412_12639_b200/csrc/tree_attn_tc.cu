@@ -11,7 +11,7 @@
 //
 // Inside a CTA (256 threads):
 //   warp 6    TMA producer: the Q tile first, then K and V tiles (bf16, 128-byte swizzle) into a
-//             5-stage ring, completion on mbarriers; the first loads are issued before anything else.
+//             3-stage ring, completion on mbarriers; the first loads are issued before anything else.
 //   warp 7    one elected lane issues tcgen05.mma (the whole warp runs the loop).  
 //             S = Q.K^T (M=128, N=64, K=128) reads Q and the K tile from shared memory; O += P.V (M=128, N=128, K=64) reads P from TMEM and the V tile from
 //             shared memory.  tcgen05.commit signals the consumers.
@@ -41,7 +41,7 @@ namespace {
 constexpr int kD = 128;
 constexpr int kBM = 128;          // query rows per CTA (TMEM lanes)
 constexpr int kBN = 64;           // keys per tile
-constexpr int kStages = 5;
+constexpr int kStages = 3;         // kPrefetch tiles in flight plus the one being consumed
 // Tiles requested ahead of the consumer.  Small on purpose: everything a CTA asks for at once
 // arrives together (the memory system serves the whole GPU's requests fairly), so a deep burst only
 // delays the first tile; the ring still lets the producer run ahead once tiles are consumed.
@@ -60,20 +60,20 @@ constexpr uint32_t kHalfTile = kBN * 128;          // 8 KB
 constexpr uint32_t kQBytes = kBM * kD * 2;          // 32 KB: two 64-column halves of 16 KB
 constexpr uint32_t kOffQ = 0;
 constexpr uint32_t kOffKV = kOffQ + kQBytes;
-constexpr uint32_t kKVBytes = kStages * 2 * kTileBytes;  // 160 KB
-// Merge: once every CTA of the cluster has left its main loop (cluster barrier), Q and the K/V ring
-// are dead and their shared memory is reused: each CTA stages its partial rows at kOffStage and
-// bulk-copies each owner's rows into that owner's merge area at kOffMrg.  A row is kMrgPitch floats:
-// 128 accumulator columns, then the row's running maximum and sum.
+constexpr uint32_t kKVBytes = kStages * 2 * kTileBytes;  // 96 KB
+// Merge: a CTA that has finished its key range stages its partial rows over its own (now idle) Q
+// tile and K/V ring and bulk-copies each owner's rows into that owner's merge area, which is
+// dedicated memory: a peer may still be in its main loop when the rows arrive.  A row is kMrgPitch
+// floats: 128 accumulator columns, then the row's running maximum and sum.
 constexpr int kMrgRows = kBM + kMaxSplits;          // rows_per * n_splits <= n_valid + n_splits - 1
 constexpr int kMrgPitch = kD + 4;                   // 528-byte rows: 16-byte accesses of 32 lanes hit all banks evenly
 constexpr uint32_t kMrgRowBytes = kMrgPitch * 4;
 constexpr uint32_t kOffStage = 0;                   // [row][kMrgPitch] staging of this CTA's partial rows
-constexpr uint32_t kOffMrg = ((kBM * kMrgRowBytes + 1023u) / 1024u) * 1024u;
+constexpr uint32_t kOffMrg = kOffKV + kKVBytes;
 constexpr uint32_t kMrgBytes = kMrgRows * kMrgRowBytes;
-constexpr uint32_t kSmemBytes = kOffKV + kKVBytes;
+constexpr uint32_t kSmemBytes = kOffMrg + kMrgBytes;
 constexpr uint32_t kSmemAlloc = kSmemBytes + 1024;  // room to align the base to 1 KB
-static_assert(kOffMrg + kMrgBytes <= kSmemBytes, "staging and merge areas must fit over Q and the K/V ring");
+static_assert(kBM * kMrgRowBytes <= kOffMrg, "staging must fit over Q and the K/V ring");
 
 // tensor memory columns (32-bit each, 128 lanes)
 constexpr uint32_t kTmemCols = 512;
@@ -337,6 +337,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   tc_fence_after();
   const uint32_t tmem_base = s_tmem_base;
   FALCON_TRACE(tid == 0, 4);
+  // Cluster phase 1: "my merge barrier exists".  Arrive now, wait just before the first remote copy.
+  if (n_splits > 1) cluster_arrive();
 
   // First loads, issued by several warps at once (a TMA instruction costs its issuing thread about
   // a hundred cycles): the producer takes the Q tile, in front so that it is not queued behind K/V,
@@ -359,7 +361,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           dev_status_or(p.status, b, FALCON_DEV_CAPACITY);
       }
       // warps 0-3: one stage each; the producer: whatever is left
-      for (int j = is_sm ? warp : 4; j < pre; j += is_sm ? kStages : 1) {
+      for (int j = is_sm ? warp : 4; j < pre; j += is_sm ? 8 : 1) {
         const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
         mbar_expect_tx(bar(kBarKVFull + j), 2 * kTileBytes);
         load_kv_tile(kdst, &tm_k, bar(kBarKVFull + j), key_begin + j * kBN, kvh, b);
@@ -375,10 +377,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     if (lane == 0) {
       for (int j = kPrefetch; j < n_my; ++j) {
         const int st = j % kStages, u = j / kStages;
-        // the next tile is requested when the oldest outstanding one has landed (and its stage is free)
-        const int jl = j - kPrefetch;
-        if (!mbar_wait(bar(kBarKVFull + jl % kStages), (jl / kStages) & 1, abort_flag)) break;
-        if (u >= 1 && !mbar_wait(bar(kBarKVEmpty + st), (u - 1) & 1, abort_flag)) break;
+        // Ramp: the stages not used yet are filled one by one as earlier tiles land (a deep first
+        // burst would only delay the first tile); after that a tile is requested as soon as its
+        // stage has been consumed, which keeps the whole ring in flight.
+        if (u == 0) {
+          const int jl = j - kPrefetch;
+          if (!mbar_wait(bar(kBarKVFull + jl % kStages), (jl / kStages) & 1, abort_flag)) break;
+        } else if (!mbar_wait(bar(kBarKVEmpty + st), (u - 1) & 1, abort_flag)) {
+          break;
+        }
         const int k0 = key_begin + j * kBN;
         const uint32_t kdst = smem_base + kOffKV + st * 2 * kTileBytes;
         const uint32_t vdst = kdst + kTileBytes;
@@ -669,10 +676,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   FALCON_TRACE(tid == 0, 72);
   if (s_abort && tid == 0) dev_status_or(p.status, b, FALCON_DEV_TIMEOUT);
   if (n_splits > 1) {
-    // Cluster phase 1: every CTA has left its main loop and staged its rows, so the merge areas
-    // (which overlay Q and the K/V ring) may be written by peers.
-    cluster_arrive();
-    cluster_wait();
+    cluster_wait();  // phase 1 (arrived long ago): every peer's merge barrier is initialised
     FALCON_TRACE(tid == 0, 73);
     if (warp == kWarpProducer && lane == 0) {
       // one bulk copy per owner: its rows of this split, contiguous in the staging area
@@ -691,43 +695,50 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const bool got = rows_mine == 0 || mbar_wait_warp(bar(kBarMrg), 0, abort_flag);
     FALCON_TRACE(tid == 0, 74);
     const float* mrg = reinterpret_cast<const float*>(smem_gen + kOffMrg);
-    for (int item = tid; got && item < rows_mine * (kD / 4); item += kTcThreads) {
-      const int rl = item / (kD / 4), c4 = item % (kD / 4);
+    for (int item = tid; got && item < rows_mine * (kD / 8); item += kTcThreads) {
+      const int rl = item / (kD / 8), c8 = item % (kD / 8);
       // all loads first (independent), then the arithmetic
       float2 m_l[kMaxSplits];
-      float4 x[kMaxSplits];
+      float4 x[kMaxSplits][2];
 #pragma unroll
       for (int s = 0; s < kMaxSplits; ++s) {
         m_l[s] = make_float2(-INFINITY, 0.f);
-        x[s] = make_float4(0.f, 0.f, 0.f, 0.f);
+        x[s][0] = x[s][1] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (s < n_splits) {
           const float* rowp = mrg + (s * rows_per + rl) * kMrgPitch;
           m_l[s] = *reinterpret_cast<const float2*>(rowp + kD);
-          x[s] = *reinterpret_cast<const float4*>(rowp + c4 * 4);
+          x[s][0] = *reinterpret_cast<const float4*>(rowp + c8 * 8);
+          x[s][1] = *reinterpret_cast<const float4*>(rowp + c8 * 8 + 4);
         }
       }
       float gm = -INFINITY;
 #pragma unroll
       for (int s = 0; s < kMaxSplits; ++s) gm = fmaxf(gm, m_l[s].x);
-      float lsum = 0.f, a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+      float lsum = 0.f, acc[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) acc[c] = 0.f;
 #pragma unroll
       for (int s = 0; s < kMaxSplits; ++s) {
         if (m_l[s].x != -INFINITY) {  // a split that saw no key of this row has no valid columns
           const float w = ex2(m_l[s].x - gm);
           lsum = fmaf(m_l[s].y, w, lsum);
-          a0 = fmaf(x[s].x, w, a0);
-          a1 = fmaf(x[s].y, w, a1);
-          a2 = fmaf(x[s].z, w, a2);
-          a3 = fmaf(x[s].w, w, a3);
+          acc[0] = fmaf(x[s][0].x, w, acc[0]);
+          acc[1] = fmaf(x[s][0].y, w, acc[1]);
+          acc[2] = fmaf(x[s][0].z, w, acc[2]);
+          acc[3] = fmaf(x[s][0].w, w, acc[3]);
+          acc[4] = fmaf(x[s][1].x, w, acc[4]);
+          acc[5] = fmaf(x[s][1].y, w, acc[5]);
+          acc[6] = fmaf(x[s][1].z, w, acc[6]);
+          acc[7] = fmaf(x[s][1].w, w, acc[7]);
         }
       }
       const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
       const int mg = mtile * kBM + row0 + rl;
-      __align__(8) __nv_bfloat162 h[2];
-      h[0] = __floats2bfloat162_rn(a0 * inv, a1 * inv);
-      h[1] = __floats2bfloat162_rn(a2 * inv, a3 * inv);
-      *reinterpret_cast<uint2*>(p.out + (static_cast<int64_t>(node_base + mg / G) * p.Hq + kvh * G + mg % G) * kD +
-                                c4 * 4) = *reinterpret_cast<const uint2*>(h);
+      __align__(16) __nv_bfloat162 h[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) h[c] = __floats2bfloat162_rn(acc[2 * c] * inv, acc[2 * c + 1] * inv);
+      *reinterpret_cast<uint4*>(p.out + (static_cast<int64_t>(node_base + mg / G) * p.Hq + kvh * G + mg % G) * kD +
+                                c8 * 8) = *reinterpret_cast<const uint4*>(h);
     }
     // Cluster phase 2: nobody leaves while a peer may still be reading its staging rows or
     // writing into its merge buffer (an owner arrives only after all its rows have landed).
