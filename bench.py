@@ -48,6 +48,23 @@ def accept_bytes(spec, tb) -> int:
     return 4 * tb.total_nodes * spec.vocab + 12 * tb.total_nodes
 
 
+def recorded_traffic(workload: str):
+    """DRAM bytes per attention launch from the committed ncu summary of this workload, or None when
+    there is none or the kernel source has changed since the counters were taken."""
+    import hashlib
+    import re
+    try:
+        text = open(os.path.join(ROOT, "profiles", "tree_attn_tc_%s_ncu.md" % workload)).read()
+        src = open(os.path.join(ROOT, "paper_2412_12639_b200", "csrc", "tree_attn_tc.cu"), "rb").read()
+    except OSError:
+        return None
+    sha = re.search(r"kernel_source_sha256:\s*([0-9a-f]{64})", text)
+    val = re.search(r"dram_bytes_per_launch:\s*(\d+)", text)
+    if not sha or not val or sha.group(1) != hashlib.sha256(src).hexdigest():
+        return None
+    return int(val.group(1))
+
+
 # --------------------------------------------------------------------------- clocks
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
@@ -168,10 +185,10 @@ def run_falcon(args):
     import torch.distributed as dist
     import paper_2412_12639_b200 as falcon
     from paper_2412_12639_b200 import binding
+    from paper_2412_12639_b200 import dist as fdist
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    info = fdist.rank_info()
+    world, rank, local = info.world, info.rank, info.local_rank
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(local)
@@ -182,8 +199,9 @@ def run_falcon(args):
 
     spec = synth.SPECS[args.workload]
     # every rank verifies its own batch of sequences (independent problems: no exchange on this path)
-    tb = synth.make_trees(spec, seed=spec.seed + rank)
-    logits_h = synth.make_logits(spec, tb, seed=spec.seed + rank)
+    seed = fdist.shard_seed(spec.seed, rank)
+    tb = synth.make_trees(spec, seed=seed)
+    logits_h = synth.make_logits(spec, tb, seed=seed)
     s_cap = synth.cache_capacity(tb)
     B, N, Hq, Hkv, D, NL = tb.batch, tb.total_nodes, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.n_layers
     scale = 1.0 / math.sqrt(D)
@@ -207,7 +225,7 @@ def run_falcon(args):
     tree_rows = [(b, int(tb.prefix_len[b]), tb.tree_size(b)) for b in range(B)]
     tkv_host = [torch.empty((NL, 2, Hkv, T, D), dtype=torch.bfloat16).pin_memory() for (_, _, T) in tree_rows]
     for layer in range(NL):
-        qh, kh, vh = synth.make_layer_qkv(spec, tb, layer, s_cap=s_cap, seed=spec.seed + rank)
+        qh, kh, vh = synth.make_layer_qkv(spec, tb, layer, s_cap=s_cap, seed=seed)
         q_host[layer] = torch.from_numpy(qh.view(np.int16)).view(torch.bfloat16)
         kt = torch.from_numpy(kh.view(np.int16)).view(torch.bfloat16)
         vt = torch.from_numpy(vh.view(np.int16)).view(torch.bfloat16)
@@ -313,12 +331,9 @@ def run_falcon(args):
         e2e_ms = e0.elapsed_time(e1)
         clocks = sampler.stop()
 
-    if world > 1:
-        t = torch.tensor([total_ms, attn_ms, e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, attn_ms, e2e_ms = (float(x) for x in t.tolist())
-    if status.any().item():
-        raise RuntimeError("device status words set: %s" % status.tolist())
+    total_ms, attn_ms, e2e_ms = fdist.max_over_ranks([total_ms, attn_ms, e2e_ms], dev)
+    if not fdist.all_ok(not status.any().item(), dev):
+        raise RuntimeError("device status words set on some rank (here: %s)" % status.tolist())
 
     h2d = (tree_host.numel() * 4 + q_host.numel() * 2 + sum(t.numel() for t in tkv_host) * 2 + logits_host.numel() * 4)
     d2h = result_host.numel() * 4
@@ -332,11 +347,7 @@ def run_falcon(args):
         pass
     peak = float(peaks.get("hbm_gbs", 6650.0))
     achieved = a_bytes / (per_launch_us * 1e-6) / 1e9
-    traffic = None
-    try:
-        traffic = json.load(open(os.path.join(ROOT, "profiles", "traffic.json"))).get(args.workload)
-    except (OSError, ValueError):
-        pass
+    traffic = recorded_traffic(args.workload)
 
     if rank != 0:
         if world > 1:
@@ -351,7 +362,7 @@ def run_falcon(args):
 
     step_bytes = NL * a_bytes + accept_bytes(spec, tb)
     line = {
-        "metric": METRIC, "value": world * 1e3 / ms_per_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": fdist.whole_job_rate(1.0, world, ms_per_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "batch": B, "n_layers": NL, "n_q_heads": Hq, "n_kv_heads": Hkv,
@@ -364,7 +375,7 @@ def run_falcon(args):
                      "frac": achieved / peak, "traffic": traffic, "bytes_per_launch": a_bytes,
                      "us_per_launch": per_launch_us,
                      "peak_source": "MEASURED_PEAKS.json hbm_gbs" if peaks else "fallback 6650 GB/s"},
-        "e2e": {"value": world * e2e_steps * 1e3 / e2e_ms, "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": fdist.whole_job_rate(e2e_steps, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h},
         "gpu_launches": args.steps * (NL + 2),
         "clocks": clocks,
