@@ -95,7 +95,8 @@ enum {
 
 struct TcParams {
   int32_t Hq, Hkv, G, s_cap, total_nodes;
-  uint32_t q_half_bytes;  // bytes of one 64-column half of the Q tile as loaded (rows of the box x 128)
+  uint32_t q_half_bytes;  // distance between the two 64-column halves of the Q tile in shared memory
+  uint32_t q_box_bytes;   // bytes one Q load brings in
   float scale_log2;
   const int32_t* node_off;
   const int32_t* parent;
@@ -224,6 +225,14 @@ constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | 
       "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr)                                                                  \
       : "memory")
 
+#define FALCON_TMEM_ST16(taddr, r)                                                                                    \
+  asm volatile(                                                                                                       \
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};" ::"r"(  \
+          r[0]),                                                                                                      \
+      "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),   \
+      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(taddr)                                          \
+      : "memory")
+
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -267,6 +276,12 @@ __device__ __forceinline__ uint64_t window64(uint64_t lo, uint64_t hi, int off) 
 }
 
 // ------------------------------------------------------------------------------------ kernel
+// kDup: the tile has at most 64 query rows.  They are then held twice, in TMEM lanes 0-63 and 64-127
+// (the Q tile is loaded twice), and the two copies share every key tile: lanes 0-63 take its key
+// columns 0-31, lanes 64-127 columns 32-63, each with its own running maximum and sum, as if they
+// were two more key splits.  All four SM sub-partitions then work on the exponentials, which is
+// what bounds a tile, instead of two.
+template <bool kDup>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const TcParams p) {
@@ -319,12 +334,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   // merge geometry: CTA `rank` owns rows [rank * rows_per, ...) of the tile
   const int rows_per = (n_valid + n_splits - 1) / n_splits;
 
-  const int n_sm_warps = (n_valid + 31) >> 5;  // softmax warps that own at least one query row
+  constexpr int kCols = kDup ? 32 : 64;  // key columns of a tile that one softmax thread handles
+  constexpr int kGroups = kDup ? 2 : 1;  // partial results per row and CTA
+  const int n_vs = kGroups * n_splits;   // partial results per row in the whole cluster
+  const bool merge = kDup || n_splits > 1;
+  const int row_warps = (n_valid + 31) >> 5;
+  const int n_sm_warps = kGroups * row_warps;  // softmax warps that own at least one query row
   const int q4 = warp & 3;
-  const int row = q4 * 32 + lane;
+  const int lane_row = q4 * 32 + lane;                       // TMEM lane, and the staging slot of its partial row
+  const int grp = kDup ? (q4 >> 1) : 0;                      // which half of a tile's key columns
+  const int row = kDup ? (q4 & 1) * 32 + lane : lane_row;    // query row of the tile
   const bool is_sm = warp < 4;
   const bool valid = is_sm && row < n_valid;
-  const bool warp_valid = is_sm && q4 * 32 < n_valid;
+  const bool warp_valid = is_sm && (row - lane) < n_valid;
 
   if (warp == kWarpProducer) {
     FALCON_TRACE(lane == 0, 1);
@@ -346,7 +368,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const uint32_t tmem_base = s_tmem_base;
   FALCON_TRACE(tid == 0, 4);
   // Cluster phase 1: "my merge barrier exists".  Arrive now, wait just before the first remote copy.
-  if (n_splits > 1) cluster_arrive();
+  if (merge) cluster_arrive();
 
   // First loads, issued by several warps at once (a TMA instruction costs its issuing thread about
   // a hundred cycles): the producer takes the Q tile, in front so that it is not queued behind K/V,
@@ -355,18 +377,30 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int pre = min(n_my, kPrefetch);
     if (lane == 0 && (is_sm || warp == kWarpProducer)) {
       if (warp == kWarpProducer) {
-        if (n_splits > 1) {
-          // this CTA will receive rows_mine rows from every split (its own included)
+        if (merge) {
+          // this CTA will receive rows_mine rows of every partial result (its own included)
           const int r0 = split * rows_per;
           const int mine = max(0, min(n_valid, r0 + rows_per) - r0);
-          mbar_expect_tx(bar(kBarMrg), static_cast<uint32_t>(n_splits * mine) * kMrgRowBytes);
+          mbar_expect_tx(bar(kBarMrg), static_cast<uint32_t>(n_vs * mine) * kMrgRowBytes);
         }
         if (n_my > 0) {
-          mbar_expect_tx(bar(kBarQ), 2 * p.q_half_bytes);
-          tma_load_5d(smem_base + kOffQ, &tm_q, bar(kBarQ), 0, 0, kvh, node_base + mtile * (kBM / G), 0);
+          const int node0 = node_base + mtile * (kBM / G);
+          if (kDup) {  // one load per 64-column half and copy; this thread takes the first copy
+            mbar_expect_tx(bar(kBarQ), 4 * p.q_box_bytes);
+            tma_load_5d(smem_base + kOffQ, &tm_q, bar(kBarQ), 0, 0, kvh, node0, 0);
+            tma_load_5d(smem_base + kOffQ + p.q_half_bytes, &tm_q, bar(kBarQ), 0, 0, kvh, node0, 1);
+          } else {
+            mbar_expect_tx(bar(kBarQ), p.q_box_bytes);
+            tma_load_5d(smem_base + kOffQ, &tm_q, bar(kBarQ), 0, 0, kvh, node0, 0);
+          }
         }
         if (split == 0 && mtile == 0 && kvh == 0 && (L + T > p.s_cap || T_real > FALCON_T_MAX))
           dev_status_or(p.status, b, FALCON_DEV_CAPACITY);
+      }
+      if (kDup && n_my > 0 && (warp == 2 || warp == 3)) {  // the second copy of the Q tile, 64 rows further down
+        const int h = warp - 2;
+        tma_load_5d(smem_base + kOffQ + h * p.q_half_bytes + 64 * 128, &tm_q, bar(kBarQ), 0, 0, kvh,
+                    node_base + mtile * (kBM / G), h);
       }
       // warps 0-3: one stage each; the producer: whatever is left
       for (int j = is_sm ? warp : 4; j < pre; j += is_sm ? 8 : 1) {
@@ -462,7 +496,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   } else if (warp_valid) {
     // ================================ softmax / correction (warps that own query rows) ================================
     const uint32_t tmem_lane = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16);
-    const int sm_tid = tid;  // softmax warps are warps 0..3
+    const int sm_idx = (grp * row_warps + (row >> 5)) * 32 + lane;  // index among the CTA's working softmax threads
 
     uint64_t anc_lo = 0, anc_hi = 0;
     if (valid) {
@@ -484,6 +518,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         anc_hi &= (nt == 64) ? 0ull : ((1ull << (nt - 64)) - 1ull);
       }
     }
+    if constexpr (kDup) {  // the key columns of the other group stay zero in this group's rows of both P buffers
+      uint32_t z[16];
+#pragma unroll
+      for (int c = 0; c < 16; ++c) z[c] = 0u;
+      FALCON_TMEM_ST16(tmem_lane + kTmemP + (grp ^ 1) * 16, z);
+      FALCON_TMEM_ST16(tmem_lane + kTmemP + 32 + (grp ^ 1) * 16, z);
+      tmem_wait_st();
+    }
     float m_used = -INFINITY, l_sum = 0.f;
     const float scale = p.scale_log2;
 
@@ -493,12 +535,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (!mbar_wait_warp(bar(kBarSFull + sb), u2 & 1, abort_flag)) break;
       FALCON_TRACE(tid == 0 && j < 6, 40 + 4 * j);
       tc_fence_after();
-      uint32_t sr[64];
-      if (warp_valid) {
-        FALCON_TMEM_LD32(tmem_lane + kTmemS + sb * kBN, sr);
-        FALCON_TMEM_LD32(tmem_lane + kTmemS + sb * kBN + 32, (sr + 32));
-        tmem_wait_ld();
-      }
+      uint32_t sr[kCols];
+      FALCON_TMEM_LD32(tmem_lane + kTmemS + sb * kBN + grp * 32, sr);
+      if constexpr (!kDup) FALCON_TMEM_LD32(tmem_lane + kTmemS + sb * kBN + 32, (sr + 32));
+      tmem_wait_ld();
       FALCON_TRACE(tid == 0 && j < 6, 41 + 4 * j);
 
       // the sequence's last tile: rows of V past the last key may hold anything (0 x NaN = NaN in the MMA)
@@ -507,39 +547,31 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int nv = S_valid - k0;  // 1..63 rows are real
         unsigned char* vtile = smem_gen + kOffKV + st * 2 * kTileBytes + kTileBytes;
         const int chunks = (kBN - nv) * 8;
-        for (int c = sm_tid; c < 2 * chunks; c += 32 * n_sm_warps) {
+        for (int c = sm_idx; c < 2 * chunks; c += 32 * n_sm_warps) {
           const int half = c / chunks, cc = c % chunks;
           *reinterpret_cast<uint4*>(vtile + half * kHalfTile + nv * 128 + cc * 16) = make_uint4(0, 0, 0, 0);
         }
         fence_async_smem();
       }
 
-      uint32_t pk[32];
+      uint32_t pk[kCols / 2];
       float alpha = 1.f;
       bool need_rescale = false;
       if (valid) {
         // scores stay raw; exp2(s * scale - m) is one FFMA + one MUFU per element (scale > 0 is
         // guaranteed by the launcher, so a maximum can be taken on the raw scores)
-        float s[64];
+        float s[kCols];
         if (k0 + kBN <= min(Lc, key_end)) {
 #pragma unroll
-          for (int c = 0; c < 64; c += 4) {
-            s[c] = __uint_as_float(sr[c]);
-            s[c + 1] = __uint_as_float(sr[c + 1]);
-            s[c + 2] = __uint_as_float(sr[c + 2]);
-            s[c + 3] = __uint_as_float(sr[c + 3]);
-          }
+          for (int c = 0; c < kCols; ++c) s[c] = __uint_as_float(sr[c]);
         } else {
           uint64_t vis = window64(anc_lo, anc_hi, k0 - Lc);
           if (key_end - k0 < kBN) vis &= (1ull << (key_end - k0)) - 1ull;  // keys of the next split
           const uint32_t vlo = static_cast<uint32_t>(vis), vhi = static_cast<uint32_t>(vis >> 32);
 #pragma unroll
-          for (int c = 0; c < 64; c += 4) {
-            const uint32_t w = c < 32 ? vlo : vhi;
+          for (int c = 0; c < kCols; ++c) {
+            const uint32_t w = kDup ? (grp ? vhi : vlo) : (c < 32 ? vlo : vhi);
             s[c] = ((w >> (c & 31)) & 1u) ? __uint_as_float(sr[c]) : -INFINITY;
-            s[c + 1] = ((w >> ((c + 1) & 31)) & 1u) ? __uint_as_float(sr[c + 1]) : -INFINITY;
-            s[c + 2] = ((w >> ((c + 2) & 31)) & 1u) ? __uint_as_float(sr[c + 2]) : -INFINITY;
-            s[c + 3] = ((w >> ((c + 3) & 31)) & 1u) ? __uint_as_float(sr[c + 3]) : -INFINITY;
           }
         }
         // One pass of exponentials against the maximum known so far.  The largest p tells whether
@@ -549,7 +581,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         auto exp_pass = [&](float neg_m) {
           pmx0 = pmx1 = add0 = add1 = add2 = add3 = 0.f;
 #pragma unroll
-          for (int c = 0; c < 32; c += 2) {
+          for (int c = 0; c < kCols / 2; c += 2) {
             const float p0 = ex2(fmaf(s[2 * c], scale, neg_m)), p1 = ex2(fmaf(s[2 * c + 1], scale, neg_m));
             const float p2 = ex2(fmaf(s[2 * c + 2], scale, neg_m)), p3 = ex2(fmaf(s[2 * c + 3], scale, neg_m));
             add0 += p0;
@@ -571,7 +603,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (redo) {
           float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-          for (int c = 0; c < 64; c += 4) {
+          for (int c = 0; c < kCols; c += 4) {
             mx0 = fmaxf(mx0, s[c]);
             mx1 = fmaxf(mx1, s[c + 1]);
             mx2 = fmaxf(mx2, s[c + 2]);
@@ -590,16 +622,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         l_sum += (add0 + add1) + (add2 + add3);
       } else {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) pk[c] = 0u;
+        for (int c = 0; c < kCols / 2; ++c) pk[c] = 0u;
       }
 
       FALCON_TRACE(tid == 0 && j < 6 && l_sum >= 0.f, 42 + 4 * j);
       // P buffer sb is free: the commit behind S(j) covers every MMA issued before it, and P.V of
       // tile j-2 was issued before Q.K^T of tile j.
 
-      FALCON_TRACE(tid == 0 && j < 6, 80 + 4 * j);
       // rare: the row maximum jumped; rescale the accumulator before this tile is added
-      if (warp_valid && __any_sync(0xffffffffu, need_rescale) && j > 0) {
+      if (__any_sync(0xffffffffu, need_rescale) && j > 0) {
         if (!mbar_wait_warp(bar(kBarPEmpty + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag)) break;
         tc_fence_after();
 #pragma unroll 1
@@ -613,12 +644,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
       }
 
-      if (warp_valid) {
+      if constexpr (kDup) {
+        FALCON_TMEM_ST16(tmem_lane + kTmemP + sb * 32 + grp * 16, pk);
+      } else {
         FALCON_TMEM_ST32(tmem_lane + kTmemP + sb * 32, pk);
-        FALCON_TRACE(tid == 0 && j < 6, 81 + 4 * j);
-        tmem_wait_st();
-        FALCON_TRACE(tid == 0 && j < 6, 82 + 4 * j);
       }
+      FALCON_TRACE(tid == 0 && j < 6, 81 + 4 * j);
+      tmem_wait_st();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(kBarPFull + sb));
@@ -626,13 +658,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       FALCON_TRACE(tid == 32 && j < 6, 107 + (j - 0));
     }
 
-    // ---- this split's partial rows: straight to global (one split) or staged for the merge ----
+    // ---- this split's partial rows: straight to global (one partial per row) or staged for the merge ----
     bool have = (n_my > 0) && !*abort_flag;
     if (have) have = mbar_wait_warp(bar(kBarODone), 0, abort_flag);
     FALCON_TRACE(tid == 0, 70);
     tc_fence_after();
     const bool write = have && valid;
-    if (n_splits == 1) {
+    if (!merge) {
       const float inv = (write && l_sum > 0.f) ? 1.f / l_sum : 0.f;
       const int mg = mtile * kBM + row;
       __nv_bfloat16* dst = p.out + (static_cast<int64_t>(node_base + mg / G) * p.Hq + kvh * G + mg % G) * kD;
@@ -655,8 +687,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
       }
     } else {
-      // Q and the K/V ring are idle now (all of this CTA's MMAs have finished): stage row -> [row][kMrgPitch]
-      float* stage = reinterpret_cast<float*>(smem_gen + kOffStage) + row * kMrgPitch;
+      // Q and the K/V ring are idle now (all of this CTA's MMAs have finished): stage lane -> [lane][kMrgPitch]
+      float* stage = reinterpret_cast<float*>(smem_gen + kOffStage) + lane_row * kMrgPitch;
       if (have) {
 #pragma unroll 1
         for (int ch = 0; ch < 2; ++ch) {
@@ -683,18 +715,22 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __syncthreads();
   FALCON_TRACE(tid == 0, 72);
   if (s_abort && tid == 0) dev_status_or(p.status, b, FALCON_DEV_TIMEOUT);
-  if (n_splits > 1) {
+  if (merge) {
     cluster_wait();  // phase 1 (arrived long ago): every peer's merge barrier is initialised
     FALCON_TRACE(tid == 0, 73);
     if (warp == kWarpProducer && lane == 0) {
-      // one bulk copy per owner: its rows of this split, contiguous in the staging area
+      // one bulk copy per owner and partial result: the owner's rows are contiguous in the staging area
       for (int o = 0; o < n_splits; ++o) {
         const int r0 = o * rows_per;
         const int cnt = min(n_valid, r0 + rows_per) - r0;
         if (cnt <= 0) break;
-        bulk_copy_to_peer(map_to_rank(smem_base + kOffMrg + static_cast<uint32_t>(split * rows_per) * kMrgRowBytes, o),
-                          smem_base + kOffStage + static_cast<uint32_t>(r0) * kMrgRowBytes,
-                          static_cast<uint32_t>(cnt) * kMrgRowBytes, map_to_rank(bar(kBarMrg), o));
+        const uint32_t peer_bar = map_to_rank(bar(kBarMrg), o);
+#pragma unroll
+        for (int g = 0; g < kGroups; ++g)
+          bulk_copy_to_peer(
+              map_to_rank(smem_base + kOffMrg + static_cast<uint32_t>((split * kGroups + g) * rows_per) * kMrgRowBytes, o),
+              smem_base + kOffStage + static_cast<uint32_t>(g * 64 + r0) * kMrgRowBytes,
+              static_cast<uint32_t>(cnt) * kMrgRowBytes, peer_bar);
       }
     }
     __syncwarp();
@@ -712,7 +748,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       for (int s = 0; s < kMaxSplits; ++s) {
         m_l[s] = make_float2(-INFINITY, 0.f);
         x[s][0] = x[s][1] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (s < n_splits) {
+        if (s < n_vs) {
           const float* rowp = mrg + (s * rows_per + rl) * kMrgPitch;
           m_l[s] = *reinterpret_cast<const float2*>(rowp + kD);
           x[s][0] = *reinterpret_cast<const float4*>(rowp + c8 * 8);
@@ -825,6 +861,7 @@ bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
 
 // Largest cluster size (number of KV splits) for which `units` clusters are co-resident.
 int pick_splits(falcon_ctx* ctx, int units, int max_tiles) {
+  // (both instantiations of the kernel have the same footprint: one CTA per SM)
   static int resident[kMaxSplits + 1] = {0};
   static std::mutex mu;
   std::lock_guard<std::mutex> lock(mu);
@@ -844,7 +881,7 @@ int pick_splits(falcon_ctx* ctx, int units, int max_tiles) {
       cfg.attrs = &attr;
       cfg.numAttrs = 1;
       int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, tree_attn_tc_kernel, &cfg) != cudaSuccess) n = -1;
+      if (cudaOccupancyMaxActiveClusters(&n, tree_attn_tc_kernel<false>, &cfg) != cudaSuccess) n = -1;
       resident[s] = n > 0 ? n : -1;
       cudaGetLastError();
     }
@@ -874,8 +911,11 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
 
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(tree_attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(kSmemAlloc));
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(tree_attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               static_cast<int>(kSmemAlloc));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaFuncSetAttribute(tree_attn_tc_kernel)");
     attr_set = true;
   }
@@ -888,8 +928,17 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   if (Hkv == 1 && kv_strides[2] == 0) kv_strides[2] = kv_strides[0] * a.s_cap;  // a size-1 dimension never strides
   if (B == 1 && kv_strides[3] == 0) kv_strides[3] = kv_strides[2] * Hkv;
   const uint32_t kv_box[5] = {64, static_cast<uint32_t>(kBN), 2, 1, 1};
+  const int max_tiles = (a.tree.max_prefix_len + a.tree.max_tree + kBN - 1) / kBN;
+  int splits = a.n_splits;
+  if (splits == 0) splits = pick_splits(ctx, Hkv * n_mtiles * B, max_tiles > 0 ? max_tiles : 1);
+  if (splits < 1) splits = 1;
+  // Trees of at most 64 query rows per KV head are held twice in the tile (two key-column groups per
+  // row), unless the cluster is so large that the merge could not take twice as many partial results.
+  const bool dup = a.tree.max_tree * G <= 64 && 2 * splits <= kMaxSplits;
+
   // q: [64, G, Hkv, N, 2]; a box is the query rows of one KV head: q_nodes nodes x G heads (at most
-  // 128 rows, a multiple of 8 so that the second half starts on a swizzle-atom boundary)
+  // 128 rows, a multiple of 8 so that the second half starts on a swizzle-atom boundary).  With two
+  // copies a box is one 64-column half of at most 64 rows, and each copy and half is its own load.
   const uint64_t row_bytes = static_cast<uint64_t>(kD) * 2;
   int q_nodes = kBM / G;
   {
@@ -900,7 +949,7 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   uint64_t q_dims[5] = {64, static_cast<uint64_t>(G), static_cast<uint64_t>(Hkv),
                         static_cast<uint64_t>(a.tree.total_nodes), 2};
   uint64_t q_strides[4] = {row_bytes, row_bytes * G, row_bytes * Hq, 128};
-  const uint32_t q_box[5] = {64, static_cast<uint32_t>(G), 1, static_cast<uint32_t>(q_nodes), 2};
+  const uint32_t q_box[5] = {64, static_cast<uint32_t>(G), 1, static_cast<uint32_t>(q_nodes), dup ? 1u : 2u};
   const CUtensorMap* tq = get_tmap(ctx, a.q, q_dims, q_strides, q_box);
   const CUtensorMap* tk = get_tmap(ctx, a.k_cache, kv_dims, kv_strides, kv_box);
   const CUtensorMap* tv = get_tmap(ctx, a.v_cache, kv_dims, kv_strides, kv_box);
@@ -910,11 +959,6 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   }
   const CUtensorMap mq = *tq, mk = *tk, mv = *tv;  // copies: later cache growth must not move what we pass
 
-  const int max_tiles = (a.tree.max_prefix_len + a.tree.max_tree + kBN - 1) / kBN;
-  int splits = a.n_splits;
-  if (splits == 0) splits = pick_splits(ctx, Hkv * n_mtiles * B, max_tiles > 0 ? max_tiles : 1);
-  if (splits < 1) splits = 1;
-
   TcParams p;
   p.Hq = Hq;
   p.Hkv = Hkv;
@@ -922,7 +966,8 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   p.s_cap = a.s_cap;
   p.total_nodes = a.tree.total_nodes;
   p.scale_log2 = a.sm_scale * kLog2e;
-  p.q_half_bytes = static_cast<uint32_t>(q_nodes) * G * 128u;
+  p.q_half_bytes = dup ? kBM * 128u : static_cast<uint32_t>(q_nodes) * G * 128u;
+  p.q_box_bytes = static_cast<uint32_t>(q_nodes) * G * 128u * (dup ? 1u : 2u);
   p.node_off = a.tree.node_off;
   p.parent = a.tree.parent;
   p.prefix_len = a.tree.prefix_len;
@@ -949,7 +994,8 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   attr.val.clusterDim.z = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, mq, mk, mv, p);
+  cudaError_t e = dup ? cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<true>, mq, mk, mv, p)
+                      : cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<false>, mq, mk, mv, p);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tree_attn_tc_kernel launch");
   return FALCON_OK;
 }
