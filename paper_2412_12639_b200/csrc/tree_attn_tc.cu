@@ -63,12 +63,12 @@ constexpr uint32_t kOffKV = kOffQ + kQBytes;
 constexpr uint32_t kKVBytes = kStages * 2 * kTileBytes;  // 96 KB
 // Merge: a CTA that has finished its key range stages its partial rows over its own (now idle) Q
 // tile and K/V ring and bulk-copies each owner's rows into that owner's merge area, which is
-// dedicated memory: a peer may still be in its main loop when the rows arrive.  A row is kMrgPitch
-// floats: 128 accumulator columns, then the row's running maximum and sum.
+// dedicated memory: a peer may still be in its main loop when the rows arrive.  A row is the 128
+// accumulator columns rounded to bf16 (the transfer between CTAs is what bounds the merge, and the
+// output is bf16 anyway), then the row's running maximum and sum in fp32, padded to kMrgRowBytes.
 constexpr int kMrgRows = kBM + kMaxSplits;          // rows_per * n_splits <= n_valid + n_splits - 1
-constexpr int kMrgPitch = kD + 4;                   // 528-byte rows: 16-byte accesses of 32 lanes hit all banks evenly
-constexpr uint32_t kMrgRowBytes = kMrgPitch * 4;
-constexpr uint32_t kOffStage = 0;                   // [row][kMrgPitch] staging of this CTA's partial rows
+constexpr uint32_t kMrgRowBytes = kD * 2 + 16;      // 272-byte rows: 16-byte accesses of 32 lanes hit all banks evenly
+constexpr uint32_t kOffStage = 0;                   // [row][kMrgRowBytes] staging of this CTA's partial rows
 constexpr uint32_t kOffMrg = kOffKV + kKVBytes;
 constexpr uint32_t kMrgBytes = kMrgRows * kMrgRowBytes;
 constexpr uint32_t kSmemBytes = kOffMrg + kMrgBytes;
@@ -687,8 +687,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
       }
     } else {
-      // Q and the K/V ring are idle now (all of this CTA's MMAs have finished): stage lane -> [lane][kMrgPitch]
-      float* stage = reinterpret_cast<float*>(smem_gen + kOffStage) + lane_row * kMrgPitch;
+      // Q and the K/V ring are idle now (all of this CTA's MMAs have finished): stage lane -> [lane][kMrgRowBytes]
+      unsigned char* stage = smem_gen + kOffStage + lane_row * kMrgRowBytes;
       if (have) {
 #pragma unroll 1
         for (int ch = 0; ch < 2; ++ch) {
@@ -698,13 +698,18 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           tmem_wait_ld();
           if (valid) {
 #pragma unroll
-            for (int c4 = 0; c4 < 16; ++c4)
-              *reinterpret_cast<uint4*>(stage + ch * 64 + c4 * 4) =
-                  make_uint4(o[4 * c4], o[4 * c4 + 1], o[4 * c4 + 2], o[4 * c4 + 3]);
+            for (int c8 = 0; c8 < 8; ++c8) {
+              __align__(16) __nv_bfloat162 h[4];
+#pragma unroll
+              for (int c = 0; c < 4; ++c)
+                h[c] = __floats2bfloat162_rn(__uint_as_float(o[8 * c8 + 2 * c]), __uint_as_float(o[8 * c8 + 2 * c + 1]));
+              *reinterpret_cast<uint4*>(stage + ch * 128 + c8 * 16) = *reinterpret_cast<const uint4*>(h);
+            }
           }
         }
       }
-      if (valid) *reinterpret_cast<float2*>(stage + kD) = make_float2(write ? m_used : -INFINITY, write ? l_sum : 0.f);
+      if (valid)
+        *reinterpret_cast<float2*>(stage + kD * 2) = make_float2(write ? m_used : -INFINITY, write ? l_sum : 0.f);
       fence_async_smem();  // the bulk copies below read these rows through the async proxy
     }
   }
@@ -738,21 +743,20 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int rows_mine = max(0, min(n_valid, row0 + rows_per) - row0);
     const bool got = rows_mine == 0 || mbar_wait_warp(bar(kBarMrg), 0, abort_flag);
     FALCON_TRACE(tid == 0, 74);
-    const float* mrg = reinterpret_cast<const float*>(smem_gen + kOffMrg);
+    const unsigned char* mrg = smem_gen + kOffMrg;
     for (int item = tid; got && item < rows_mine * (kD / 8); item += kTcThreads) {
       const int rl = item / (kD / 8), c8 = item % (kD / 8);
       // all loads first (independent), then the arithmetic
       float2 m_l[kMaxSplits];
-      float4 x[kMaxSplits][2];
+      uint4 x[kMaxSplits];  // 8 bf16 columns of each partial row
 #pragma unroll
       for (int s = 0; s < kMaxSplits; ++s) {
         m_l[s] = make_float2(-INFINITY, 0.f);
-        x[s][0] = x[s][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        x[s] = make_uint4(0u, 0u, 0u, 0u);
         if (s < n_vs) {
-          const float* rowp = mrg + (s * rows_per + rl) * kMrgPitch;
-          m_l[s] = *reinterpret_cast<const float2*>(rowp + kD);
-          x[s][0] = *reinterpret_cast<const float4*>(rowp + c8 * 8);
-          x[s][1] = *reinterpret_cast<const float4*>(rowp + c8 * 8 + 4);
+          const unsigned char* rowp = mrg + static_cast<uint32_t>(s * rows_per + rl) * kMrgRowBytes;
+          m_l[s] = *reinterpret_cast<const float2*>(rowp + kD * 2);
+          x[s] = *reinterpret_cast<const uint4*>(rowp + c8 * 16);
         }
       }
       float gm = -INFINITY;
@@ -766,14 +770,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (m_l[s].x != -INFINITY) {  // a split that saw no key of this row has no valid columns
           const float w = ex2(m_l[s].x - gm);
           lsum = fmaf(m_l[s].y, w, lsum);
-          acc[0] = fmaf(x[s][0].x, w, acc[0]);
-          acc[1] = fmaf(x[s][0].y, w, acc[1]);
-          acc[2] = fmaf(x[s][0].z, w, acc[2]);
-          acc[3] = fmaf(x[s][0].w, w, acc[3]);
-          acc[4] = fmaf(x[s][1].x, w, acc[4]);
-          acc[5] = fmaf(x[s][1].y, w, acc[5]);
-          acc[6] = fmaf(x[s][1].z, w, acc[6]);
-          acc[7] = fmaf(x[s][1].w, w, acc[7]);
+          const uint32_t xs[4] = {x[s].x, x[s].y, x[s].z, x[s].w};
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {  // a bf16 is the upper half of the fp32 of the same value
+            acc[2 * c] = fmaf(__uint_as_float(xs[c] << 16), w, acc[2 * c]);
+            acc[2 * c + 1] = fmaf(__uint_as_float(xs[c] & 0xffff0000u), w, acc[2 * c + 1]);
+          }
         }
       }
       const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
