@@ -11,7 +11,7 @@
 //
 // Inside a CTA (256 threads):
 //   warp 6    TMA producer: the Q tile first, then K and V tiles (bf16, 128-byte swizzle) into a
-//             3-stage ring, completion on mbarriers; the first loads are issued before anything else.
+//             4-stage ring, completion on mbarriers; the first loads are issued before anything else.
 //   warp 7    one elected lane issues tcgen05.mma (the whole warp runs the loop).  
 //             S = Q.K^T (M=128, N=64, K=128) reads Q and the K tile from shared memory; O += P.V (M=128, N=128, K=64) reads P from TMEM and the V tile from
 //             shared memory.  tcgen05.commit signals the consumers.
@@ -41,7 +41,7 @@ namespace {
 constexpr int kD = 128;
 constexpr int kBM = 128;          // query rows per CTA (TMEM lanes)
 constexpr int kBN = 64;           // keys per tile
-constexpr int kStages = 3;         // kPrefetch tiles in flight plus the one being consumed
+constexpr int kStages = 4;         // ring depth: what shared memory leaves room for next to Q and the merge area
 // Tiles requested ahead of the consumer.  Small on purpose: everything a CTA asks for at once
 // arrives together (the memory system serves the whole GPU's requests fairly), so a deep burst only
 // delays the first tile; the ring still lets the producer run ahead once tiles are consumed.
@@ -60,7 +60,7 @@ constexpr uint32_t kHalfTile = kBN * 128;          // 8 KB
 constexpr uint32_t kQBytes = kBM * kD * 2;          // 32 KB: two 64-column halves of 16 KB
 constexpr uint32_t kOffQ = 0;
 constexpr uint32_t kOffKV = kOffQ + kQBytes;
-constexpr uint32_t kKVBytes = kStages * 2 * kTileBytes;  // 96 KB
+constexpr uint32_t kKVBytes = kStages * 2 * kTileBytes;  // 128 KB
 // Merge: a CTA that has finished its key range stages its partial rows over its own (now idle) Q
 // tile and K/V ring and bulk-copies each owner's rows into that owner's merge area, which is
 // dedicated memory: a peer may still be in its main loop when the rows arrive.  A row is the 128
@@ -377,11 +377,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int pre = min(n_my, kPrefetch);
     if (lane == 0 && (is_sm || warp == kWarpProducer)) {
       if (warp == kWarpProducer) {
-        if (merge) {
-          // this CTA will receive rows_mine rows of every partial result (its own included)
+        if (n_splits > 1) {
+          // this CTA will receive rows_mine rows of every other CTA's partial results
           const int r0 = split * rows_per;
           const int mine = max(0, min(n_valid, r0 + rows_per) - r0);
-          mbar_expect_tx(bar(kBarMrg), static_cast<uint32_t>(n_vs * mine) * kMrgRowBytes);
+          mbar_expect_tx(bar(kBarMrg), static_cast<uint32_t>((n_vs - kGroups) * mine) * kMrgRowBytes);
         }
         if (n_my > 0) {
           const int node0 = node_base + mtile * (kBM / G);
@@ -724,11 +724,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     cluster_wait();  // phase 1 (arrived long ago): every peer's merge barrier is initialised
     FALCON_TRACE(tid == 0, 73);
     if (warp == kWarpProducer && lane == 0) {
-      // one bulk copy per owner and partial result: the owner's rows are contiguous in the staging area
+      // one bulk copy per other owner and partial result: the owner's rows are contiguous in the
+      // staging area (this CTA's own rows are merged from there directly)
       for (int o = 0; o < n_splits; ++o) {
         const int r0 = o * rows_per;
         const int cnt = min(n_valid, r0 + rows_per) - r0;
         if (cnt <= 0) break;
+        if (o == split) continue;
         const uint32_t peer_bar = map_to_rank(bar(kBarMrg), o);
 #pragma unroll
         for (int g = 0; g < kGroups; ++g)
@@ -741,9 +743,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     __syncwarp();
     const int row0 = split * rows_per;
     const int rows_mine = max(0, min(n_valid, row0 + rows_per) - row0);
-    const bool got = rows_mine == 0 || mbar_wait_warp(bar(kBarMrg), 0, abort_flag);
+    const bool got = rows_mine == 0 || n_splits == 1 || mbar_wait_warp(bar(kBarMrg), 0, abort_flag);
     FALCON_TRACE(tid == 0, 74);
     const unsigned char* mrg = smem_gen + kOffMrg;
+    const unsigned char* own = smem_gen + kOffStage + static_cast<uint32_t>(row0) * kMrgRowBytes;
     for (int item = tid; got && item < rows_mine * (kD / 8); item += kTcThreads) {
       const int rl = item / (kD / 8), c8 = item % (kD / 8);
       // all loads first (independent), then the arithmetic
@@ -754,7 +757,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         m_l[s] = make_float2(-INFINITY, 0.f);
         x[s] = make_uint4(0u, 0u, 0u, 0u);
         if (s < n_vs) {
-          const unsigned char* rowp = mrg + static_cast<uint32_t>(s * rows_per + rl) * kMrgRowBytes;
+          const unsigned char* rowp = (s / kGroups == split)
+                                          ? own + static_cast<uint32_t>((s % kGroups) * 64 + rl) * kMrgRowBytes
+                                          : mrg + static_cast<uint32_t>(s * rows_per + rl) * kMrgRowBytes;
           m_l[s] = *reinterpret_cast<const float2*>(rowp + kD * 2);
           x[s] = *reinterpret_cast<const uint4*>(rowp + c8 * 16);
         }
