@@ -296,11 +296,30 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int kvh = blockIdx.y % p.Hkv, mtile = blockIdx.y / p.Hkv, b = blockIdx.z;
   const int G = p.G;
 
-  if (tid == 0) {
-    prefetch_tmap(&tm_q);
-    prefetch_tmap(&tm_k);
-    prefetch_tmap(&tm_v);
+  // What touches no global memory comes first: tensor-map prefetch, barrier initialisation (all but
+  // the two whose count depends on the tree), tensor memory.  Under programmatic dependent launch
+  // this part runs while the previous kernel of the stream is still finishing.
+  const uint32_t bars = smem_u32(s_bars);
+  auto bar = [&](int i) { return bars + 8u * static_cast<uint32_t>(i); };
+  if (warp == kWarpProducer) {
+    if (lane == 0) {
+      s_abort = 0;
+      prefetch_tmap(&tm_q);
+      prefetch_tmap(&tm_k);
+      prefetch_tmap(&tm_v);
+    }
+    if (lane < kNumBars && lane != kBarPFull && lane != kBarPFull + 1) mbar_init(bar(lane), 1);  // barrier i: lane i
+  } else if (warp == kWarpMma) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  // Everything below may read what earlier kernels of the stream wrote (tree arrays, q, the tree's
+  // K/V rows) and writes `out`: wait until they have completed.  Then let the next kernel's CTAs
+  // be scheduled as this grid's CTAs leave their SMs (a no-op without programmatic launch).
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   int node_base, T_real, L_raw;
   if (p.have_host) {
     node_base = p.h_node_off[b];
@@ -313,7 +332,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   }
   const int T = min(T_real, FALCON_T_MAX);
   const int rows_total = T * G;
-  if (mtile * kBM >= rows_total) return;  // same decision in every CTA of the cluster
+  if (mtile * kBM >= rows_total) {  // no query rows here; same decision in every CTA of the cluster
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kWarpMma) {
+      tc_fence_after();
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(s_tmem_base), "r"(kTmemCols) : "memory");
+    }
+    return;
+  }
   const int n_valid = min(kBM, rows_total - mtile * kBM);
   const int L = max(L_raw, 0);
   const int Lc = min(L, p.s_cap);
@@ -327,8 +354,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t bars = smem_u32(s_bars);
-  auto bar = [&](int i) { return bars + 8u * static_cast<uint32_t>(i); };
   volatile int* abort_flag = &s_abort;
 
   // merge geometry: CTA `rank` owns rows [rank * rows_per, ...) of the tile
@@ -350,17 +375,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   if (warp == kWarpProducer) {
     FALCON_TRACE(lane == 0, 1);
-    if (lane == 0) s_abort = 0;
-    if (lane < kNumBars) {  // barrier i is initialised by lane i
-      const bool per_warp = lane == kBarPFull || lane == kBarPFull + 1;
-      mbar_init(bar(lane), per_warp ? n_sm_warps : 1);
-    }
+    if (lane == kBarPFull || lane == kBarPFull + 1) mbar_init(bar(lane), n_sm_warps);  // one arrival per softmax warp
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  } else if (warp == kWarpMma) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
-                 "r"(kTmemCols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
@@ -994,13 +1010,17 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   cfg.blockDim = dim3(kTcThreads);
   cfg.dynamicSmemBytes = kSmemAlloc;
   cfg.stream = s;
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeClusterDimension;
-  attr.val.clusterDim.x = splits;
-  attr.val.clusterDim.y = 1;
-  attr.val.clusterDim.z = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = splits;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  // Programmatic dependent launch: this grid may be scheduled while the previous kernel of the stream
+  // drains; the kernel itself waits for that kernel's completion before it touches global memory.
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
   cudaError_t e = dup ? cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<true>, mq, mk, mv, p)
                       : cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<false>, mq, mk, mv, p);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tree_attn_tc_kernel launch");
