@@ -46,9 +46,9 @@ constexpr int kStages = 4;         // ring depth: what shared memory leaves room
 // arrives together (the memory system serves the whole GPU's requests fairly), so a deep burst only
 // delays the first tile; the ring still lets the producer run ahead once tiles are consumed.
 constexpr int kPrefetch = 2;
-constexpr int kTcThreads = 256;    // warps 0-3 softmax (TMEM quadrant = warp), 4-5 idle, 6 producer, 7 MMA
-constexpr int kWarpProducer = 6;
-constexpr int kWarpMma = 7;
+constexpr int kTcThreads = 320;    // warps 0-7 softmax (TMEM quadrant = warp % 4, stream = warp / 4), 8 producer, 9 MMA
+constexpr int kWarpProducer = 8;
+constexpr int kWarpMma = 9;
 constexpr int kMaxSplits = 8;
 constexpr int kHostSeqs = 8;
 constexpr uint32_t kSpinLimit = 1u << 18;
@@ -77,9 +77,9 @@ static_assert(kBM * kMrgRowBytes <= kOffMrg, "staging must fit over Q and the K/
 
 // tensor memory columns (32-bit each, 128 lanes)
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kTmemO = 0;      // 128 columns: fp32 accumulator
-constexpr uint32_t kTmemS = 128;    // 2 x 64 columns: fp32 scores
-constexpr uint32_t kTmemP = 256;    // 2 x 32 columns: bf16 pairs
+constexpr uint32_t kTmemO = 0;      // 2 x 128 columns: fp32 accumulators (one per softmax stream)
+constexpr uint32_t kTmemS = 256;    // 2 x 64 columns: fp32 scores
+constexpr uint32_t kTmemP = 384;    // 2 x 32 columns: bf16 pairs
 
 enum {
   kBarQ = 0,                         // the Q tile has landed in shared memory
@@ -289,6 +289,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __shared__ __align__(8) uint64_t s_bars[kNumBars];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
+  __shared__ float2 s_ml[2][kBM];  // [stream][row]: running maximum and sum, exchanged once after the loop
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   FALCON_TRACE(tid == 0, 0);
@@ -361,6 +362,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   constexpr int kCols = kDup ? 32 : 64;  // key columns of a tile that one softmax thread handles
   constexpr int kGroups = kDup ? 2 : 1;  // partial results per row and CTA
+  // Softmax streams: with two, warps 0-3 take the even tiles of the CTA's run and warps 4-7 the odd
+  // ones, each stream with its own maximum, sum and accumulator.  Warps w and w+4 sit on the same
+  // scheduler and reach the same TMEM lanes, so one stream's exponentials fill the gaps of the
+  // other's loads, stores and barrier traffic, and after the loop the two threads of a row fold
+  // the two accumulators into one partial result at no extra traffic.
+  constexpr int kStreams = kDup ? 1 : 2;
   const int n_vs = kGroups * n_splits;   // partial results per row in the whole cluster
   const bool merge = kDup || n_splits > 1;
   const int row_warps = (n_valid + 31) >> 5;
@@ -369,7 +376,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int lane_row = q4 * 32 + lane;                       // TMEM lane, and the staging slot of its partial row
   const int grp = kDup ? (q4 >> 1) : 0;                      // which half of a tile's key columns
   const int row = kDup ? (q4 & 1) * 32 + lane : lane_row;    // query row of the tile
-  const bool is_sm = warp < 4;
+  const bool is_sm = warp < 4 * kStreams;
+  const bool is_ld = warp < 4;                               // warps that issue one of the first loads
+  const int strm = kStreams == 2 ? ((warp >> 2) & 1) : 0;
   const bool valid = is_sm && row < n_valid;
   const bool warp_valid = is_sm && (row - lane) < n_valid;
 
@@ -391,7 +400,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   // and the last stage; lane 0 of warps 0-3 takes stages 0-3.
   {
     const int pre = min(n_my, kPrefetch);
-    if (lane == 0 && (is_sm || warp == kWarpProducer)) {
+    if (lane == 0 && (is_ld || warp == kWarpProducer)) {
       if (warp == kWarpProducer) {
         if (n_splits > 1) {
           // this CTA will receive rows_mine rows of every other CTA's partial results
@@ -419,7 +428,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     node_base + mtile * (kBM / G), h);
       }
       // warps 0-3: one stage each; the producer: whatever is left
-      for (int j = is_sm ? warp : 4; j < pre; j += is_sm ? 8 : 1) {
+      for (int j = is_ld ? warp : 4; j < pre; j += is_ld ? 8 : 1) {
         const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
         mbar_expect_tx(bar(kBarKVFull + j), 2 * kTileBytes);
         load_kv_tile(kdst, &tm_k, bar(kBarKVFull + j), key_begin + j * kBN, kvh, b);
@@ -461,33 +470,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
       bool ok = mbar_wait_warp(bar(kBarQ), 0, abort_flag);
       FALCON_TRACE(elected, 5);
-      auto issue_pv = [&](int t) -> bool {
-        const int st = t % kStages, pb = t & 1;
-        FALCON_TRACE(elected && t < 6, 113 + (t - 0));
-        if (!mbar_wait_warp(bar(kBarPFull + pb), (t >> 1) & 1, abort_flag)) return false;
-        FALCON_TRACE(elected && t < 6, 12 + 4 * t);
-        tc_fence_after();
-        const uint32_t vbase = smem_base + kOffKV + st * 2 * kTileBytes + kTileBytes;
-        if (elected) {
-#pragma unroll
-          for (int kk = 0; kk < kBN / 16; ++kk) {
-            // P: 16 keys = 8 packed columns; V: MN-major, 16 keys = 2 KB, the two 64-column halves 8 KB apart
-            const uint64_t bd = smem_desc(vbase + kk * 2048, kHalfTile, 1024);
-            umma_bf16_ts(tmem_base + kTmemO, tmem_base + kTmemP + pb * 32 + kk * 8, bd, kIdescPV,
-                         (t > 0 || kk > 0) ? 1u : 0u);
-          }
-          umma_commit(bar(kBarKVEmpty + st));
-          umma_commit(bar(kBarPEmpty + pb));
-          FALCON_TRACE(t < 6, 13 + 4 * t);
-        }
-        __syncwarp();
-        return true;
-      };
-      for (int j = 0; ok && j < n_my; ++j) {
+      auto issue_qk = [&](int j) -> bool {
         const int st = j % kStages, sb = j & 1;
-        // S buffer sb held the scores of tile j-2; the softmax warps read them before they wrote
-        // P(j-2), and P(j-2) was waited for before P.V of tile j-2 was issued: it is free.
-        if (!mbar_wait_warp(bar(kBarKVFull + st), (j / kStages) & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_wait_warp(bar(kBarKVFull + st), (j / kStages) & 1, abort_flag)) return false;
         FALCON_TRACE(elected && j < 6, 10 + 4 * j);
         tc_fence_after();
         const uint32_t kbase = smem_base + kOffKV + st * 2 * kTileBytes;
@@ -503,9 +488,40 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           FALCON_TRACE(j < 6, 11 + 4 * j);
         }
         __syncwarp();
-        if (j >= 1 && !issue_pv(j - 1)) { ok = false; break; }
+        return true;
+      };
+      auto issue_pv = [&](int t) {
+        const int st = t % kStages, pb = t & 1;
+        const uint32_t vbase = smem_base + kOffKV + st * 2 * kTileBytes + kTileBytes;
+        const uint32_t acc = tmem_base + kTmemO + (kStreams == 2 ? pb * kD : 0);
+        if (elected) {
+#pragma unroll
+          for (int kk = 0; kk < kBN / 16; ++kk) {
+            // P: 16 keys = 8 packed columns; V: MN-major, 16 keys = 2 KB, the two 64-column halves 8 KB apart
+            const uint64_t bd = smem_desc(vbase + kk * 2048, kHalfTile, 1024);
+            umma_bf16_ts(acc, tmem_base + kTmemP + pb * 32 + kk * 8, bd, kIdescPV, (t >= kStreams || kk > 0) ? 1u : 0u);
+          }
+          umma_commit(bar(kBarKVEmpty + st));
+          umma_commit(bar(kBarPEmpty + pb));
+          FALCON_TRACE(t < 6, 13 + 4 * t);
+        }
+        __syncwarp();
+      };
+      // Two tiles of scores are always in flight (one per S buffer).  When P(t) is there, S buffer
+      // t & 1 has been read, so Q.K^T of tile t+2 can go into it.  It is issued after P.V of tile t:
+      // the commit behind S(t+2) then also covers that P.V, which is what tells the softmax warps
+      // that P buffer t & 1 may be overwritten.
+      ok = ok && issue_qk(0);
+      if (ok && n_my > 1) ok = issue_qk(1);
+      for (int t = 0; ok && t < n_my; ++t) {
+        const int pb = t & 1;
+        FALCON_TRACE(elected && t < 6, 113 + (t - 0));
+        if (!mbar_wait_warp(bar(kBarPFull + pb), (t >> 1) & 1, abort_flag)) { ok = false; break; }
+        FALCON_TRACE(elected && t < 6, 12 + 4 * t);
+        tc_fence_after();
+        issue_pv(t);
+        if (t + 2 < n_my) ok = issue_qk(t + 2);
       }
-      if (ok) ok = issue_pv(n_my - 1);
       if (elected) umma_commit(bar(kBarODone));  // fires once every MMA issued so far has finished
       __syncwarp();
     }
@@ -545,7 +561,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     float m_used = -INFINITY, l_sum = 0.f;
     const float scale = p.scale_log2;
 
-    for (int j = 0; j < n_my; ++j) {
+    const uint32_t tmem_acc = tmem_lane + kTmemO + strm * kD;  // this stream's accumulator
+    for (int j = strm; j < n_my; j += kStreams) {
       const int sb = j & 1, u2 = j >> 1, st = j % kStages;
       const int k0 = key_begin + j * kBN;
       if (!mbar_wait_warp(bar(kBarSFull + sb), u2 & 1, abort_flag)) break;
@@ -645,18 +662,20 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       // P buffer sb is free: the commit behind S(j) covers every MMA issued before it, and P.V of
       // tile j-2 was issued before Q.K^T of tile j.
 
-      // rare: the row maximum jumped; rescale the accumulator before this tile is added
-      if (__any_sync(0xffffffffu, need_rescale) && j > 0) {
-        if (!mbar_wait_warp(bar(kBarPEmpty + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag)) break;
+      // rare: the row maximum jumped; rescale the accumulator before this tile is added (the
+      // stream's previous tile must have been added first)
+      if (__any_sync(0xffffffffu, need_rescale) && j >= kStreams) {
+        const int jp = j - kStreams;
+        if (!mbar_wait_warp(bar(kBarPEmpty + (jp & 1)), (jp >> 1) & 1, abort_flag)) break;
         tc_fence_after();
 #pragma unroll 1
         for (int ch = 0; ch < 4; ++ch) {
           uint32_t o[32];
-          FALCON_TMEM_LD32(tmem_lane + kTmemO + ch * 32, o);
+          FALCON_TMEM_LD32(tmem_acc + ch * 32, o);
           tmem_wait_ld();
 #pragma unroll
           for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-          FALCON_TMEM_ST32(tmem_lane + kTmemO + ch * 32, o);
+          FALCON_TMEM_ST32(tmem_acc + ch * 32, o);
         }
       }
 
@@ -671,7 +690,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(kBarPFull + sb));
       FALCON_TRACE(tid == 0 && j < 6, 43 + 4 * j);
-      FALCON_TRACE(tid == 32 && j < 6, 107 + (j - 0));
+      FALCON_TRACE(tid == 128 && j < 6, 107 + (j - 0));
     }
 
     // ---- this split's partial rows: straight to global (one partial per row) or staged for the merge ----
@@ -680,6 +699,63 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     FALCON_TRACE(tid == 0, 70);
     tc_fence_after();
     const bool write = have && valid;
+    if constexpr (kStreams == 2) {
+      // Fold the two streams' accumulators: the two threads of a row (same lanes, so each reaches
+      // both accumulators) swap their maximum and sum, then each takes 64 of the 128 columns.
+      s_ml[strm][row] = make_float2(m_used, l_sum);
+      asm volatile("bar.sync %0, 64;" ::"r"(1 + q4) : "memory");
+      const float2 ot = s_ml[strm ^ 1][row];
+      const float gm = fmaxf(m_used, ot.x);
+      const float w_me = (m_used == -INFINITY) ? 0.f : ex2(m_used - gm);
+      const float w_ot = (ot.x == -INFINITY) ? 0.f : ex2(ot.x - gm);
+      const float l_row = l_sum * w_me + ot.y * w_ot;
+      const float w0 = strm == 0 ? w_me : w_ot, w1 = strm == 0 ? w_ot : w_me;  // weights of accumulators 0 and 1
+      const float inv = merge ? 1.f : ((write && l_row > 0.f) ? 1.f / l_row : 0.f);
+      const int mg = mtile * kBM + row;
+      __nv_bfloat16* dst =
+          p.out + (static_cast<int64_t>(node_base + mg / G) * p.Hq + kvh * G + mg % G) * kD + strm * 64;
+      unsigned char* stage = smem_gen + kOffStage + lane_row * kMrgRowBytes + strm * 128;
+#pragma unroll 1
+      for (int ch = 0; ch < 2; ++ch) {
+        uint32_t o0[32], o1[32];
+        if (have) {
+          FALCON_TMEM_LD32(tmem_lane + kTmemO + strm * 64 + ch * 32, o0);
+          FALCON_TMEM_LD32(tmem_lane + kTmemO + kD + strm * 64 + ch * 32, o1);
+          tmem_wait_ld();
+        }
+        if (valid) {
+#pragma unroll
+          for (int c8 = 0; c8 < 4; ++c8) {
+            __align__(16) __nv_bfloat162 h[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              const int i = 8 * c8 + 2 * c;
+              // an accumulator that no tile was added to holds anything: it is skipped, not scaled by 0
+              float a = 0.f, bq = 0.f;
+              if (write && w0 > 0.f) {
+                a = __uint_as_float(o0[i]) * w0;
+                bq = __uint_as_float(o0[i + 1]) * w0;
+              }
+              if (write && w1 > 0.f) {
+                a = fmaf(__uint_as_float(o1[i]), w1, a);
+                bq = fmaf(__uint_as_float(o1[i + 1]), w1, bq);
+              }
+              h[c] = __floats2bfloat162_rn(a * inv, bq * inv);
+            }
+            if (merge)
+              *reinterpret_cast<uint4*>(stage + ch * 64 + c8 * 16) = *reinterpret_cast<const uint4*>(h);
+            else
+              *reinterpret_cast<uint4*>(dst + ch * 32 + c8 * 8) = *reinterpret_cast<const uint4*>(h);
+          }
+        }
+      }
+      if (merge) {
+        if (valid && strm == 0)
+          *reinterpret_cast<float2*>(smem_gen + kOffStage + lane_row * kMrgRowBytes + kD * 2) =
+              make_float2(write ? gm : -INFINITY, write ? l_row : 0.f);
+        fence_async_smem();  // the bulk copies below read these rows through the async proxy
+      }
+    } else
     if (!merge) {
       const float inv = (write && l_sum > 0.f) ? 1.f / l_sum : 0.f;
       const int mg = mtile * kBM + row;
