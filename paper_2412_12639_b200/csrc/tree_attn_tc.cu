@@ -709,45 +709,49 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const float w_me = (m_used == -INFINITY) ? 0.f : ex2(m_used - gm);
       const float w_ot = (ot.x == -INFINITY) ? 0.f : ex2(ot.x - gm);
       const float l_row = l_sum * w_me + ot.y * w_ot;
-      const float w0 = strm == 0 ? w_me : w_ot, w1 = strm == 0 ? w_ot : w_me;  // weights of accumulators 0 and 1
-      const float inv = merge ? 1.f : ((write && l_row > 0.f) ? 1.f / l_row : 0.f);
+      const float inv = merge ? 1.f : (l_row > 0.f ? 1.f / l_row : 0.f);
+      // weights of accumulators 0 and 1, normalisation folded in
+      const float f0 = (strm == 0 ? w_me : w_ot) * inv, f1 = (strm == 0 ? w_ot : w_me) * inv;
+      // Accumulator 1 holds anything when the CTA's run is a single tile; otherwise both are finite
+      // (a row whose keys were all masked in a stream has weight 0 and an all-zero accumulator).
+      const bool two = n_my > 1;
       const int mg = mtile * kBM + row;
       __nv_bfloat16* dst =
           p.out + (static_cast<int64_t>(node_base + mg / G) * p.Hq + kvh * G + mg % G) * kD + strm * 64;
       unsigned char* stage = smem_gen + kOffStage + lane_row * kMrgRowBytes + strm * 128;
+      if (have) {
 #pragma unroll 1
-      for (int ch = 0; ch < 2; ++ch) {
-        uint32_t o0[32], o1[32];
-        if (have) {
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t o0[32], o1[32];
           FALCON_TMEM_LD32(tmem_lane + kTmemO + strm * 64 + ch * 32, o0);
-          FALCON_TMEM_LD32(tmem_lane + kTmemO + kD + strm * 64 + ch * 32, o1);
+          if (two) FALCON_TMEM_LD32(tmem_lane + kTmemO + kD + strm * 64 + ch * 32, o1);
           tmem_wait_ld();
-        }
-        if (valid) {
+          if (valid) {
+            uint32_t h[16];
+            if (two) {
 #pragma unroll
-          for (int c8 = 0; c8 < 4; ++c8) {
-            __align__(16) __nv_bfloat162 h[4];
+              for (int c = 0; c < 16; ++c) {
+                const float a = fmaf(__uint_as_float(o1[2 * c]), f1, __uint_as_float(o0[2 * c]) * f0);
+                const float bq = fmaf(__uint_as_float(o1[2 * c + 1]), f1, __uint_as_float(o0[2 * c + 1]) * f0);
+                const __nv_bfloat162 hh = __floats2bfloat162_rn(a, bq);
+                h[c] = *reinterpret_cast<const uint32_t*>(&hh);
+              }
+            } else {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              const int i = 8 * c8 + 2 * c;
-              // an accumulator that no tile was added to holds anything: it is skipped, not scaled by 0
-              float a = 0.f, bq = 0.f;
-              if (write && w0 > 0.f) {
-                a = __uint_as_float(o0[i]) * w0;
-                bq = __uint_as_float(o0[i + 1]) * w0;
+              for (int c = 0; c < 16; ++c) {
+                const __nv_bfloat162 hh =
+                    __floats2bfloat162_rn(__uint_as_float(o0[2 * c]) * f0, __uint_as_float(o0[2 * c + 1]) * f0);
+                h[c] = *reinterpret_cast<const uint32_t*>(&hh);
               }
-              if (write && w1 > 0.f) {
-                a = fmaf(__uint_as_float(o1[i]), w1, a);
-                bq = fmaf(__uint_as_float(o1[i + 1]), w1, bq);
-              }
-              h[c] = __floats2bfloat162_rn(a * inv, bq * inv);
             }
-            if (merge)
-              *reinterpret_cast<uint4*>(stage + ch * 64 + c8 * 16) = *reinterpret_cast<const uint4*>(h);
-            else
-              *reinterpret_cast<uint4*>(dst + ch * 32 + c8 * 8) = *reinterpret_cast<const uint4*>(h);
+            uint4* d4 = merge ? reinterpret_cast<uint4*>(stage + ch * 64) : reinterpret_cast<uint4*>(dst + ch * 32);
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) d4[c4] = make_uint4(h[4 * c4], h[4 * c4 + 1], h[4 * c4 + 2], h[4 * c4 + 3]);
           }
         }
+      } else if (valid && !merge) {  // nothing was computed (a wait ran out): the row reads as zero
+#pragma unroll
+        for (int c4 = 0; c4 < 8; ++c4) reinterpret_cast<uint4*>(dst)[c4] = make_uint4(0u, 0u, 0u, 0u);
       }
       if (merge) {
         if (valid && strm == 0)
