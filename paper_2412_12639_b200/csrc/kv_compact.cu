@@ -3,7 +3,10 @@
 // of one (layer, K|V, sequence, KV head): it reads every source row into
 // registers, passes a barrier, then writes, so a destination row that is also an
 // earlier source row (in-place mode) cannot be clobbered before it is read.
-// Launch/latency-bound byte copy with 16-byte accesses.
+// Launch/latency-bound byte copy with 16-byte accesses: what matters is that the
+// whole grid is resident at once (each CTA is a chain of three dependent round
+// trips to memory), so trees small enough get a variant that keeps few registers
+// per thread and moves K and V in the same CTA.
 #include "common.cuh"
 
 namespace falcon {
@@ -11,6 +14,7 @@ namespace {
 
 constexpr int kCompactThreads = 256;
 constexpr int kMaxChunksPerThread = 16;  // 128 rows x 32 chunks (D = 256) / 256 threads
+constexpr int kSmallChunksPerThread = 4; // the small variant: trees of up to 1024 chunks per matrix
 
 struct CompactParams {
   int32_t batch, n_layers, n_kv_heads, head_dim, s_cap, path_stride;
@@ -27,12 +31,19 @@ struct CompactParams {
   int32_t* new_len;
 };
 
+// kBoth: blockIdx.z is the layer and the CTA moves K then V (both held in registers at once);
+// otherwise blockIdx.z is 2 * layer + (0 for K, 1 for V).
+template <int kChunks, bool kBoth>
 __global__ void __launch_bounds__(kCompactThreads) kv_compact_kernel(const CompactParams p) {
   __shared__ int s_path[FALCON_T_MAX];
   __shared__ int s_bad;
+  // Under programmatic dependent launch the grid may start while the previous kernel of the stream
+  // drains: nothing is read or written before that kernel has completed.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int h = blockIdx.x, b = blockIdx.y;
-  const int layer = blockIdx.z >> 1, is_v = blockIdx.z & 1;
+  const int layer = kBoth ? blockIdx.z : (blockIdx.z >> 1);
   const int tid = threadIdx.x;
+  constexpr int kMats = kBoth ? 2 : 1;
 
   const int base = p.node_off[b];
   const int T = p.node_off[b + 1] - base;
@@ -42,6 +53,9 @@ __global__ void __launch_bounds__(kCompactThreads) kv_compact_kernel(const Compa
   int fault = 0;
   if (T < 1 || T > FALCON_T_MAX || n < 1 || n > T) fault |= FALCON_DEV_BAD_PATH;
   if (L < 0 || L + (separate ? n : T) > p.s_cap) fault |= FALCON_DEV_CAPACITY;
+  // the variant was picked from the caller's max_tree: a longer path than it can hold is refused
+  if (n > 0 && static_cast<int64_t>(n) * (p.head_dim >> 3) > static_cast<int64_t>(kChunks) * kCompactThreads)
+    fault |= FALCON_DEV_CAPACITY;
   if (tid == 0) s_bad = 0;
   __syncthreads();
   if (!fault && tid < n) {
@@ -51,7 +65,7 @@ __global__ void __launch_bounds__(kCompactThreads) kv_compact_kernel(const Compa
   }
   __syncthreads();
   if (s_bad) fault |= FALCON_DEV_BAD_PATH;
-  const bool first = (h == 0 && blockIdx.z == 0 && tid == 0);
+  const bool first = (h == 0 && blockIdx.z == 0 && tid == 0);  // one writer of the new length per sequence
   if (fault) {  // leave the cache alone, report, keep the old length
     if (first) {
       dev_status_or(p.status, b, fault);
@@ -61,33 +75,43 @@ __global__ void __launch_bounds__(kCompactThreads) kv_compact_kernel(const Compa
   }
   if (first) p.new_len[b] = L + n;
 
-  __nv_bfloat16* cache = static_cast<__nv_bfloat16*>(is_v ? p.v_layers[layer] : p.k_layers[layer]) +
-                         b * p.stride_b + h * p.stride_h;
-  const __nv_bfloat16* tree = nullptr;
-  if (separate)
-    tree = static_cast<const __nv_bfloat16*>(is_v ? p.v_tree_layers[layer] : p.k_tree_layers[layer]);
+  __nv_bfloat16* cache[kMats];
+  const __nv_bfloat16* tree[kMats];
+#pragma unroll
+  for (int m = 0; m < kMats; ++m) {
+    const bool is_v = kBoth ? (m == 1) : ((blockIdx.z & 1) != 0);
+    cache[m] = static_cast<__nv_bfloat16*>(is_v ? p.v_layers[layer] : p.k_layers[layer]) + b * p.stride_b + h * p.stride_h;
+    tree[m] = separate ? static_cast<const __nv_bfloat16*>(is_v ? p.v_tree_layers[layer] : p.k_tree_layers[layer])
+                       : nullptr;
+  }
 
   const int cpr = p.head_dim >> 3;  // 16-byte chunks per row
   const int total = n * cpr;
-  uint4 regs[kMaxChunksPerThread];
+  uint4 regs[kMats][kChunks];
 #pragma unroll
-  for (int k = 0; k < kMaxChunksPerThread; ++k) {
-    const int idx = tid + k * kCompactThreads;
-    if (idx < total) {
-      const int j = idx / cpr, c = idx - j * cpr;
-      const __nv_bfloat16* src =
-          separate ? tree + (static_cast<int64_t>(base + s_path[j]) * p.n_kv_heads + h) * p.head_dim
-                   : cache + static_cast<int64_t>(L + s_path[j]) * p.stride_s;
-      regs[k] = *reinterpret_cast<const uint4*>(src + 8 * c);
+  for (int m = 0; m < kMats; ++m) {
+#pragma unroll
+    for (int k = 0; k < kChunks; ++k) {
+      const int idx = tid + k * kCompactThreads;
+      if (idx < total) {
+        const int j = idx / cpr, c = idx - j * cpr;
+        const __nv_bfloat16* src =
+            separate ? tree[m] + (static_cast<int64_t>(base + s_path[j]) * p.n_kv_heads + h) * p.head_dim
+                     : cache[m] + static_cast<int64_t>(L + s_path[j]) * p.stride_s;
+        regs[m][k] = *reinterpret_cast<const uint4*>(src + 8 * c);
+      }
     }
   }
   __syncthreads();  // every source row is in registers before any destination row is written
 #pragma unroll
-  for (int k = 0; k < kMaxChunksPerThread; ++k) {
-    const int idx = tid + k * kCompactThreads;
-    if (idx < total) {
-      const int j = idx / cpr, c = idx - j * cpr;
-      *reinterpret_cast<uint4*>(cache + static_cast<int64_t>(L + j) * p.stride_s + 8 * c) = regs[k];
+  for (int m = 0; m < kMats; ++m) {
+#pragma unroll
+    for (int k = 0; k < kChunks; ++k) {
+      const int idx = tid + k * kCompactThreads;
+      if (idx < total) {
+        const int j = idx / cpr, c = idx - j * cpr;
+        *reinterpret_cast<uint4*>(cache[m] + static_cast<int64_t>(L + j) * p.stride_s + 8 * c) = regs[m][k];
+      }
     }
   }
 }
@@ -116,9 +140,24 @@ int launch_kv_compact(falcon_ctx* ctx, const falcon_compact_args& a, cudaStream_
   p.path = a.path;
   p.n_path = a.n_path;
   p.new_len = a.new_len;
-  dim3 grid(a.n_kv_heads, a.tree.batch, 2 * a.n_layers);
-  kv_compact_kernel<<<grid, kCompactThreads, 0, s>>>(p);
-  cudaError_t e = cudaGetLastError();
+  // the path is at most max_tree rows long: small trees take the variant with K and V in one CTA
+  const int64_t max_chunks = static_cast<int64_t>(a.tree.max_tree) * (a.head_dim >> 3);
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(kCompactThreads);
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaError_t e;
+  if (max_chunks <= static_cast<int64_t>(kSmallChunksPerThread) * kCompactThreads) {
+    cfg.gridDim = dim3(a.n_kv_heads, a.tree.batch, a.n_layers);
+    e = cudaLaunchKernelEx(&cfg, kv_compact_kernel<kSmallChunksPerThread, true>, p);
+  } else {
+    cfg.gridDim = dim3(a.n_kv_heads, a.tree.batch, 2 * a.n_layers);
+    e = cudaLaunchKernelEx(&cfg, kv_compact_kernel<kMaxChunksPerThread, false>, p);
+  }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "kv_compact_kernel launch");
   return FALCON_OK;
 }

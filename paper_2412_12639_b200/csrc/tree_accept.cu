@@ -54,10 +54,24 @@ __global__ void __launch_bounds__(kAcceptThreads) tree_accept_kernel(const Accep
   __shared__ int s_par[FALCON_T_MAX], s_tok[FALCON_T_MAX], s_g[FALCON_T_MAX];
   __shared__ int s_key[kAcceptThreads / 32];
 
+  // Under programmatic dependent launch the grid may start while the previous kernel of the stream
+  // drains: nothing is read or written before that kernel has completed.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int row = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x;
   const int c0 = chunk * p.chunk_len;
   const int c1 = min(p.vocab, c0 + p.chunk_len);
   const float* rowp = p.logits + static_cast<int64_t>(row) * p.logits_stride;
+
+  // sequence that owns this row (looked up first: its loads overlap the scan below)
+  int lo = 0, hi = p.batch;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (p.node_off[mid] <= row) lo = mid; else hi = mid;
+  }
+  const int b = lo;
+  const int base = p.node_off[b];
+  const int T_real = p.node_off[b + 1] - base;
+  const int T = min(T_real, FALCON_T_MAX);
 
   Best mine{-INFINITY, kNone};
   if (c0 < c1) {
@@ -88,17 +102,6 @@ __global__ void __launch_bounds__(kAcceptThreads) tree_accept_kernel(const Accep
   if ((tid & 31) == 0) warp_best[tid >> 5] = mine;
   __syncthreads();
 
-  // sequence that owns this row
-  int lo = 0, hi = p.batch;
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (p.node_off[mid] <= row) lo = mid; else hi = mid;
-  }
-  const int b = lo;
-  const int base = p.node_off[b];
-  const int T_real = p.node_off[b + 1] - base;
-  const int T = min(T_real, FALCON_T_MAX);
-
   if (tid == 0) {
     Best r = warp_best[0];
 #pragma unroll
@@ -118,7 +121,18 @@ __global__ void __launch_bounds__(kAcceptThreads) tree_accept_kernel(const Accep
   if (tid < T) {
     Best r{-INFINITY, kNone};
     const int64_t o = static_cast<int64_t>(base + tid) * p.chunks;
-    for (int c = 0; c < p.chunks; ++c) r = merge(r, Best{__ldcg(p.part_val + o + c), __ldcg(p.part_idx + o + c)});
+    for (int c0f = 0; c0f < p.chunks; c0f += 8) {  // eight partials in flight: the loads are independent
+      float v[8];
+      int ix[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const bool in = c0f + k < p.chunks;
+        v[k] = in ? __ldcg(p.part_val + o + c0f + k) : -INFINITY;
+        ix[k] = in ? __ldcg(p.part_idx + o + c0f + k) : kNone;
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) r = merge(r, Best{v[k], ix[k]});
+    }
     const int g = (r.i == kNone) ? 0 : r.i;
     p.argmax_out[base + tid] = g;
     s_g[tid] = g;
@@ -210,9 +224,16 @@ int launch_tree_accept(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_
   p.part_idx = reinterpret_cast<int32_t*>(static_cast<float*>(ctx->ws) + part);
   p.tickets = ctx->tickets;
 
-  dim3 grid(chunks, N);
-  tree_accept_kernel<<<grid, kAcceptThreads, 0, s>>>(p);
-  cudaError_t e = cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(chunks, N);
+  cfg.blockDim = dim3(kAcceptThreads);
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, tree_accept_kernel, p);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tree_accept_kernel launch");
   return FALCON_OK;
 }
