@@ -436,6 +436,55 @@ def test_compact_bad_path_or_capacity_leaves_cache_untouched():
     np.testing.assert_array_equal(gv[0][1], vs[0][1])
 
 
+def test_compact_path_longer_than_the_declared_max_tree_is_refused():
+    """The launcher picks the copy variant from the caller's max_tree; a sequence whose path does not
+    fit that variant is reported (capacity) and its cache is left alone, the other sequence is compacted."""
+    rng = np.random.default_rng(6)
+    tb = H.make_trees([100, 8], [10, 3], rng, parents=[synth.chain_tree(100), synth.chain_tree(8)])
+    path = np.full((2, 128), -1, np.int32)
+    path[0, :80] = np.arange(80)                       # 80 rows x 16 chunks = 1280 > 1024: too long for the small variant
+    path[1, :5] = np.arange(5)
+    n_path = np.array([80, 5], np.int32)
+    s_cap = 112
+    ks = [rng.integers(0, 65536, size=(2, 2, s_cap, 128)).astype(np.uint16)]
+    vs = [rng.integers(0, 65536, size=(2, 2, s_cap, 128)).astype(np.uint16)]
+    dt = H.DevTrees(tb)
+    honest = dt.desc
+
+    def understated(**kw):
+        d = honest(**kw)
+        d.max_tree = 60                                 # passes the host check (60 x 2 >= 108 nodes), still too small
+        return d
+
+    dt.desc = understated
+    gk, gv, new_len = H.run_compact(dt, 2, 128, ks, vs, path, n_path)
+    st = dt.status.cpu().numpy()
+    assert st[0] & binding.DEV_CAPACITY and st[1] == 0
+    assert new_len.tolist() == [10, 8]
+    np.testing.assert_array_equal(gk[0][0], ks[0][0])
+    np.testing.assert_array_equal(gv[0][0], vs[0][0])
+    ref_k, ref_v = ks[0].copy(), vs[0].copy()
+    for ref in (ref_k, ref_v):
+        oracle.kv_compact(tb.node_off, tb.prefix_len, 2, 128, ref, strides_of(ref), s_cap, path, n_path)
+    np.testing.assert_array_equal(gk[0][1, :, :8], ref_k[1, :, :8])
+    np.testing.assert_array_equal(gv[0][1, :, :8], ref_v[1, :, :8])
+
+
+@pytest.mark.parametrize("T,G,L,splits", [(60, 1, 700, 1), (60, 1, 700, 4), (32, 2, 100, 2), (17, 1, 0, 1),
+                                           (80, 1, 30, 2), (80, 1, 500, 1), (128, 1, 64, 3), (16, 8, 1000, 5)])
+def test_attn_tc_row_arrangements(T, G, L, splits):
+    """Both arrangements of the tensor-core kernel (two copies of at most 64 rows; two streams on
+    alternate tiles, including runs of a single tile where the second stream has nothing) at forced splits."""
+    rng = np.random.default_rng(100 * T + 10 * G + splits)
+    Hkv = 2
+    tb, q, k, v = random_case(rng, [T], [L], Hkv * G, Hkv, 128, slack=1)
+    ref = oracle_attn(tb, Hkv * G, Hkv, 128, q, k, v)
+    out, rc = H.run_attn(H.DevTrees(tb), Hkv * G, Hkv, 128, q, k, v, kernel=binding.ATTN_TC, n_splits=splits,
+                         check=False)
+    tc_or_skip(rc)
+    H.assert_attn_close(out, ref, tb.node_off)
+
+
 # ------------------------------------------------------------------------ ABI
 def test_abi_rejects_bad_arguments_without_launching():
     rng = np.random.default_rng(1)
