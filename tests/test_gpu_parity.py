@@ -485,6 +485,31 @@ def test_attn_tc_row_arrangements(T, G, L, splits):
     H.assert_attn_close(out, ref, tb.node_off)
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_attn_tc_random_batches_and_splits(seed):
+    """Random batches (ragged trees and prefixes around the tile edges), head groupings and forced
+    splits through the tensor-core kernel: oracle parity, bit-identical reruns, clean status words."""
+    rng = np.random.default_rng(9000 + seed)
+    for _ in range(6):
+        G = int(rng.choice([1, 2, 4, 8]))
+        Hkv = int(rng.choice([1, 2, 3]))
+        B = int(rng.choice([1, 2, 3]))
+        sizes = [int(rng.integers(1, 129)) for _ in range(B)]
+        prefs = [int(rng.choice([0, 1, 63, 64, 65, int(rng.integers(0, 400))])) for _ in range(B)]
+        splits = int(rng.choice([0, 1, 2, 3, 4, 5, 8]))
+        tb, q, k, v = random_case(rng, sizes, prefs, Hkv * G, Hkv, 128, slack=int(rng.integers(0, 4)))
+        ref = oracle_attn(tb, Hkv * G, Hkv, 128, q, k, v)
+        dt = H.DevTrees(tb)
+        hc = bool(rng.integers(0, 2))
+        out, rc = H.run_attn(dt, Hkv * G, Hkv, 128, q, k, v, kernel=binding.ATTN_TC, n_splits=splits, check=False,
+                             host_copies=hc)
+        tc_or_skip(rc)
+        H.assert_attn_close(out, ref, tb.node_off)
+        again, _ = H.run_attn(dt, Hkv * G, Hkv, 128, q, k, v, kernel=binding.ATTN_TC, n_splits=splits, host_copies=hc)
+        np.testing.assert_array_equal(out, again)
+        assert not dt.status.cpu().numpy().any()
+
+
 # ------------------------------------------------------------------------ ABI
 def test_abi_rejects_bad_arguments_without_launching():
     rng = np.random.default_rng(1)
