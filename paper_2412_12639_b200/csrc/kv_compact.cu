@@ -15,6 +15,7 @@ namespace {
 constexpr int kCompactThreads = 256;
 constexpr int kMaxChunksPerThread = 16;  // 128 rows x 32 chunks (D = 256) / 256 threads
 constexpr int kSmallChunksPerThread = 4; // the small variant: trees of up to 1024 chunks per matrix
+constexpr int kMidChunksPerThread = 6;   // up to 1536 chunks per matrix (96 nodes at head_dim 128)
 
 struct CompactParams {
   int32_t batch, n_layers, n_kv_heads, head_dim, s_cap, path_stride;
@@ -154,6 +155,9 @@ int launch_kv_compact(falcon_ctx* ctx, const falcon_compact_args& a, cudaStream_
   if (max_chunks <= static_cast<int64_t>(kSmallChunksPerThread) * kCompactThreads) {
     cfg.gridDim = dim3(a.n_kv_heads, a.tree.batch, a.n_layers);
     e = cudaLaunchKernelEx(&cfg, kv_compact_kernel<kSmallChunksPerThread, true>, p);
+  } else if (max_chunks <= static_cast<int64_t>(kMidChunksPerThread) * kCompactThreads) {
+    cfg.gridDim = dim3(a.n_kv_heads, a.tree.batch, a.n_layers);
+    e = cudaLaunchKernelEx(&cfg, kv_compact_kernel<kMidChunksPerThread, true>, p);
   } else {
     cfg.gridDim = dim3(a.n_kv_heads, a.tree.batch, 2 * a.n_layers);
     e = cudaLaunchKernelEx(&cfg, kv_compact_kernel<kMaxChunksPerThread, false>, p);
