@@ -9,18 +9,23 @@
 // and every CTA normalises and stores its share of the rows.  No partial result
 // touches global memory.
 //
-// Inside a CTA (256 threads):
-//   warp 6    TMA producer: the Q tile first, then K and V tiles (bf16, 128-byte swizzle) into a
-//             4-stage ring, completion on mbarriers; the first loads are issued before anything else.
-//   warp 7    one elected lane issues tcgen05.mma (the whole warp runs the loop).  
-//             S = Q.K^T (M=128, N=64, K=128) reads Q and the K tile from shared memory; O += P.V (M=128, N=128, K=64) reads P from TMEM and the V tile from
-//             shared memory.  tcgen05.commit signals the consumers.
-//   warps 0-3 one thread per query row (warps 4-5 only pad the CTA so that the two service
-//             warps sit on other schedulers than the first two softmax warps):
-//             per tile tcgen05.ld of the score row, tree mask from the node's ancestor bit
-//             set, online softmax with a lazily updated maximum (the accumulator is
-//             rescaled only when a weight would exceed 2^8), P written back
-//             to TMEM as packed bf16.
+// Inside a CTA (320 threads):
+//   warp 8    TMA producer: the Q tile first, then K and V tiles (bf16, 128-byte swizzle) into a
+//             4-stage ring, completion on mbarriers; the first loads are issued by several warps.
+//   warp 9    one elected lane issues tcgen05.mma (the whole warp runs the loop).
+//             S = Q.K^T (M=128, N=64, K=128) reads Q and the K tile from shared memory;
+//             O += P.V (M=128, N=128, K=64) reads P from TMEM and the V tile from shared memory.
+//             tcgen05.commit signals the consumers.
+//   warps 0-7 softmax, one thread per (query row, stream or copy): per tile tcgen05.ld of the
+//             score row, tree mask from the node's ancestor bit set, online softmax with a lazily
+//             updated maximum (the accumulator is rescaled only when a weight would exceed 2^8),
+//             P written back to TMEM as packed bf16.  Units of more than 64 rows run two streams
+//             (warps 0-3 the even tiles, 4-7 the odd ones, one accumulator each, folded at the
+//             end); units of at most 64 rows hold the rows twice (lanes 0-63 and 64-127) and give
+//             each copy half of every tile's key columns (warps 0-3 only).
+// The partial rows cross the cluster as bf16 columns plus fp32 (max, sum).  All three falcon
+// kernels are launched programmatically dependent: set-up that touches no global memory runs
+// before griddepcontrol.wait and overlaps the previous kernel's drain.
 // Every mbarrier wait is bounded; a wait that runs out sets FALCON_DEV_TIMEOUT in the
 // status word, and the CTA still reaches the cluster barrier and frees its TMEM.
 #include <cuda.h>
