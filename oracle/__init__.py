@@ -95,6 +95,20 @@ def argmax(logits, vocab=None, n_threads=0):
     return g
 
 
+def topm(logits, m, vocab=None, n_threads=0):
+    """logits: C-contiguous fp32 [N, stride].  Returns (values [N, m] fp32, indices [N, m] int32), best first."""
+    assert logits.dtype == np.float32 and logits.ndim == 2 and logits.flags.c_contiguous
+    N, stride = logits.shape
+    V = stride if vocab is None else vocab
+    val = np.empty((N, m), dtype=np.float32)
+    idx = np.empty((N, m), dtype=np.int32)
+    rc = lib().oracle_topm(_p(logits, C.c_float), C.c_int32(N), C.c_int32(V), C.c_int64(stride), C.c_int32(m),
+                           _p(val, C.c_float), _p(idx, C.c_int32), C.c_int(n_threads))
+    if rc:
+        raise ValueError("oracle_topm failed: %d" % rc)
+    return val, idx
+
+
 def _accept(fn, node_off, parent, token, g, path_stride):
     node_off, parent, token, g = _i32(node_off), _i32(parent), _i32(token), _i32(g)
     B = len(node_off) - 1

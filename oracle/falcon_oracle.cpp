@@ -17,6 +17,8 @@
 //     length is the tau of Section 4.2.
 //   * compaction: "record the accepted tokens and their corresponding features
 //     for the subsequent drafting phase" (Section 3.4), in its KV-cache form.
+//   * top-m selection (the step before verification): every tree node is expanded
+//     with the m most probable tokens of the drafter's distribution (Appendix A).
 //
 // Every routine is the plain definition: visible sets by walking parent
 // pointers, two-pass softmax with double accumulators, sequential argmax scan,
@@ -248,6 +250,40 @@ int oracle_argmax(const float* logits, int32_t N, int32_t V, int64_t stride, int
         idx = v;
       }
     g[i] = idx;
+  }
+  return 0;
+}
+
+// Top-m entries of every row, best first: the children a tree node is given when the tree is
+// grown ("the m tokens with the highest probability", Appendix A; m = 20 at the root there).
+// Plain definition: m passes over the row, each taking the best entry not taken yet.  Order:
+// larger value first, the lower index among equal values (+0 and -0 are equal); a NaN counts as
+// -inf and is reported as -inf.  Needs 1 <= m <= V.
+int oracle_topm(const float* logits, int32_t N, int32_t V, int64_t stride, int32_t m, float* top_val,
+                int32_t* top_idx, int n_threads) {
+  if (N < 0 || V < 1 || stride < V || m < 1 || m > V) return 1;
+  const int nt = pick_threads(n_threads);
+  (void)nt;
+#pragma omp parallel for num_threads(nt)
+  for (int32_t i = 0; i < N; ++i) {
+    const float* row = logits + static_cast<int64_t>(i) * stride;
+    std::vector<char> taken(static_cast<size_t>(V), 0);
+    for (int32_t r = 0; r < m; ++r) {
+      const float ninf = -std::numeric_limits<float>::infinity();
+      float best = ninf;
+      int32_t idx = -1;
+      for (int32_t v = 0; v < V; ++v) {
+        if (taken[v]) continue;
+        const float x = (row[v] != row[v]) ? ninf : row[v];
+        if (idx < 0 || x > best) {  // strict: the first (lowest) index among equals stays
+          best = x;
+          idx = v;
+        }
+      }
+      taken[idx] = 1;
+      top_val[static_cast<int64_t>(i) * m + r] = best;
+      top_idx[static_cast<int64_t>(i) * m + r] = idx;
+    }
   }
   return 0;
 }

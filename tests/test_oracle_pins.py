@@ -479,3 +479,57 @@ def test_bf16_bit_conversion_round_trip_and_rounding():
     y = np.random.default_rng(0).standard_normal(10000).astype(np.float32)
     np.testing.assert_array_equal(synth.f32_to_bf16_bits(y),
                                   torch.from_numpy(y).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16))
+
+
+# ------------------------------------------------------------------ top-m selection (Appendix A)
+def test_topm_matches_a_stable_library_sort():
+    # second opinion: numpy's stable argsort of the negated row gives the same order (lower index first among equals)
+    rng = np.random.default_rng(3)
+    for V, m in ((1, 1), (7, 7), (1000, 20), (32001, 20), (4099, 32)):
+        x = rng.standard_normal((4, V)).astype(np.float32)
+        x[:, ::5] = np.round(x[:, ::5])                       # plenty of exact ties
+        val, idx = oracle.topm(x, m)
+        ref = np.argsort(-x, axis=1, kind="stable")[:, :m]
+        np.testing.assert_array_equal(idx, ref)
+        np.testing.assert_array_equal(val, np.take_along_axis(x, ref, 1))
+
+
+def test_topm_with_torch_topk_values_and_first_entry_is_argmax():
+    rng = np.random.default_rng(4)
+    x = rng.standard_normal((6, 5000)).astype(np.float32)
+    val, idx = oracle.topm(x, 20)
+    tv, _ = torch.topk(torch.from_numpy(x), 20, dim=1)        # values are unique up to ties; indices may differ on ties
+    np.testing.assert_array_equal(val, tv.numpy())
+    np.testing.assert_array_equal(idx[:, 0], oracle.argmax(x))
+
+
+def test_topm_hand_worked_ties_zero_signs_and_nan():
+    # row: values              index: 0    1     2    3     4    5        6
+    x = np.array([[1.0, 3.0, 3.0, -0.0, 0.0, np.nan, -np.inf]], np.float32)
+    val, idx = oracle.topm(x, 7)
+    # 3 (index 1 before 2), 1, then the zeros as equals (index 3 before 4), then -inf entries by index: the NaN at 5
+    # counts as -inf and comes before the real -inf at 6
+    assert idx[0].tolist() == [1, 2, 0, 3, 4, 5, 6]
+    assert val[0, :3].tolist() == [3.0, 3.0, 1.0] and np.all(val[0, 3:5] == 0.0)
+    assert np.isneginf(val[0, 5]) and np.isneginf(val[0, 6])
+    # a descending row returns 0..m-1, an ascending one V-1..V-m
+    d = np.arange(50, 0, -1, dtype=np.float32)[None]
+    assert oracle.topm(d, 5)[1][0].tolist() == [0, 1, 2, 3, 4]
+    assert oracle.topm(d[:, ::-1].copy(), 5)[1][0].tolist() == [49, 48, 47, 46, 45]
+    with pytest.raises(ValueError):
+        oracle.topm(d, 51)
+
+
+def test_topm_respects_row_stride_and_permutations():
+    rng = np.random.default_rng(5)
+    V, stride, m = 777, 800, 12
+    buf = rng.standard_normal((3, stride)).astype(np.float32)
+    buf[:, V:] = 100.0                                         # padding must never be selected
+    val, idx = oracle.topm(buf, m, vocab=V)
+    assert idx.max() < V
+    perm = rng.permutation(V)
+    shuffled = buf.copy()
+    shuffled[:, :V] = buf[:, :V][:, perm]
+    val2, idx2 = oracle.topm(shuffled, m, vocab=V)
+    np.testing.assert_array_equal(val, val2)                   # the values are a property of the multiset
+    np.testing.assert_array_equal(perm[idx2], idx)             # distinct values almost surely: indices map back
