@@ -159,6 +159,34 @@ typedef struct {
 int falcon_tree_accept(falcon_ctx* ctx, const falcon_accept_args* args, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * falcon_topm - the m best entries of every logits row, best first: the children
+ * a node of the decoding tree is given when the tree is grown (Appendix A: "the m
+ * tokens with the highest probability", m = 20 at the root).  It is the step just
+ * before verification and scans the same kind of [rows, vocab] fp32 matrix as
+ * the acceptance call.
+ *
+ *   order      larger value first; the lower index among equal values (+0 == -0);
+ *              a NaN counts as -inf and is reported as -inf
+ *   top_val    [n_rows, m] fp32, top_idx [n_rows, m] int32, row-major, device memory
+ *   limits     1 <= m <= min(vocab, FALCON_TOPM_MAX); vocab <= 262144;
+ *              n_rows <= 65535; logits 4-byte aligned
+ * Errors: FALCON_ERR_INVALID_ARG / FALCON_ERR_CAPACITY, nothing launched.  Scratch
+ * comes from the context (the first call of a size allocates it).
+ * ------------------------------------------------------------------------- */
+#define FALCON_TOPM_MAX 32
+typedef struct {
+  int32_t n_rows;
+  int32_t vocab;
+  int64_t logits_stride;  /* elements between rows, >= vocab                          */
+  const float* logits;    /* fp32 [n_rows, logits_stride]                             */
+  int32_t m;
+  float* top_val;         /* [n_rows, m]                                              */
+  int32_t* top_idx;       /* [n_rows, m]                                              */
+} falcon_topm_args;
+
+int falcon_topm(falcon_ctx* ctx, const falcon_topm_args* args, void* stream);
+
+/* ---------------------------------------------------------------------------
  * falcon_tree_accept_static - falcon_tree_accept for callers that cannot allocate
  * device memory.  (The paper has no counterpart: this is a deployment variant of
  * the call above, same arguments, same results.)

@@ -8,4 +8,4 @@ is independent of the library.
 """
 from . import binding, synth  # noqa: F401
 from .binding import (ATTN_AUTO, ATTN_SIMT, ATTN_TC, Context, FalconError, accept_args, attn_args,  # noqa: F401
-                      compact_args, tree_desc)
+                      compact_args, topm_args, tree_desc)

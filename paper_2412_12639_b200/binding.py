@@ -48,6 +48,11 @@ class AcceptArgs(C.Structure):
                 ("n_path", C.c_void_p), ("next_token", C.c_void_p)]
 
 
+class TopmArgs(C.Structure):
+    _fields_ = [("n_rows", C.c_int32), ("vocab", C.c_int32), ("logits_stride", C.c_int64), ("logits", C.c_void_p),
+                ("m", C.c_int32), ("top_val", C.c_void_p), ("top_idx", C.c_void_p)]
+
+
 class CompactArgs(C.Structure):
     _fields_ = [("tree", TreeDesc), ("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("k_cache_layers", C.c_void_p), ("v_cache_layers", C.c_void_p), ("kv_stride_b", C.c_int64),
@@ -79,7 +84,7 @@ def load_library():
     lib.falcon_tree_validate_host.argtypes = [C.c_void_p, C.c_int32]
     lib.falcon_tree_validate_host.restype = C.c_int
     for name, argt in (("falcon_tree_attn", AttnArgs), ("falcon_tree_accept", AcceptArgs),
-                       ("falcon_kv_compact", CompactArgs)):
+                       ("falcon_kv_compact", CompactArgs), ("falcon_topm", TopmArgs)):
         fn = getattr(lib, name)
         fn.argtypes = [C.c_void_p, C.POINTER(argt), C.c_void_p]
         fn.restype = C.c_int
@@ -101,6 +106,7 @@ def falcon_tree_validate_host(parent) -> int:
 
 
 STATIC_MAX_NODES, STATIC_MAX_BATCH = 1024, 256
+TOPM_MAX = 32
 
 
 def falcon_tree_accept_static(args: "AcceptArgs", stream=None, check: bool = True) -> int:
@@ -178,6 +184,12 @@ class Context:
             self._check(rc, "falcon_tree_accept")
         return rc
 
+    def falcon_topm(self, args: TopmArgs, stream=None, check: bool = True) -> int:
+        rc = self._lib.falcon_topm(self._h, C.byref(args), _stream(stream))
+        if check:
+            self._check(rc, "falcon_topm")
+        return rc
+
     def falcon_kv_compact(self, args: CompactArgs, stream=None, check: bool = True) -> int:
         rc = self._lib.falcon_kv_compact(self._h, C.byref(args), _stream(stream))
         if check:
@@ -196,6 +208,10 @@ def accept_args(tree: TreeDesc, vocab, logits, logits_stride, argmax_out, path, 
                 next_token) -> AcceptArgs:
     return AcceptArgs(tree, vocab, logits_stride, _ptr(logits), _ptr(argmax_out), _ptr(path), path_stride,
                       _ptr(n_path), _ptr(next_token))
+
+
+def topm_args(n_rows, vocab, logits, logits_stride, m, top_val, top_idx) -> TopmArgs:
+    return TopmArgs(n_rows, vocab, logits_stride, _ptr(logits), m, _ptr(top_val), _ptr(top_idx))
 
 
 def compact_args(tree: TreeDesc, n_layers, n_kv_heads, head_dim, k_cache_layers, v_cache_layers, strides, s_cap,

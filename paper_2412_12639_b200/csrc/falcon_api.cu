@@ -150,6 +150,16 @@ int falcon_tree_accept(falcon_ctx* ctx, const falcon_accept_args* a, void* strea
   return launch_tree_accept(ctx, *a, static_cast<cudaStream_t>(stream));
 }
 
+int falcon_topm(falcon_ctx* ctx, const falcon_topm_args* a, void* stream) {
+  if (!ctx || !a) return FALCON_ERR_INVALID_ARG;
+  if (!a->logits || !a->top_val || !a->top_idx) return FALCON_ERR_INVALID_ARG;
+  if (a->n_rows < 1 || a->vocab < 1 || a->logits_stride < a->vocab) return FALCON_ERR_INVALID_ARG;
+  if (a->m < 1 || a->m > a->vocab || a->m > FALCON_TOPM_MAX) return FALCON_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(a->logits) & 3) return FALCON_ERR_INVALID_ARG;
+  if (a->vocab > 64 * 4096) return FALCON_ERR_CAPACITY;
+  return launch_tree_topm(ctx, *a, static_cast<cudaStream_t>(stream));
+}
+
 int falcon_kv_compact(falcon_ctx* ctx, const falcon_compact_args* a, void* stream) {
   if (!ctx || !a) return FALCON_ERR_INVALID_ARG;
   int rc = check_tree_desc(a->tree, false);

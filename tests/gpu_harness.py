@@ -120,6 +120,18 @@ def run_accept(dt: DevTrees, logits: np.ndarray, vocab=None, path_stride=128):
     return g.cpu().numpy(), path.cpu().numpy(), n_path.cpu().numpy(), nxt.cpu().numpy()
 
 
+def run_topm(logits: np.ndarray, m, vocab=None, check=True):
+    """logits fp32 [N, stride] -> (values [N, m], indices [N, m], rc)."""
+    ld = torch.from_numpy(np.ascontiguousarray(logits)).cuda()
+    N, stride = ld.shape
+    V = stride if vocab is None else vocab
+    val = torch.full((N, m), float("nan"), dtype=torch.float32, device="cuda")
+    idx = torch.full((N, m), -7, dtype=torch.int32, device="cuda")
+    rc = ctx().falcon_topm(binding.topm_args(N, V, ld, stride, m, val, idx), check=check)
+    torch.cuda.synchronize()
+    return val.cpu().numpy(), idx.cpu().numpy(), rc
+
+
 def run_compact(dt: DevTrees, Hkv, D, k_layers, v_layers, path, n_path, k_tree_layers=None, v_tree_layers=None,
                 s_cap=None):
     """k_layers / v_layers: lists of uint16 [B,Hkv,s_cap,D] host arrays.  Returns compacted copies and new_len."""

@@ -510,6 +510,58 @@ def test_attn_tc_random_batches_and_splits(seed):
         assert not dt.status.cpu().numpy().any()
 
 
+# ----------------------------------------------------------------------- top-m
+@pytest.mark.parametrize("N,V,stride,m", [(1, 1, 1, 1), (3, 7, 9, 7), (5, 1000, 1000, 20), (60, 32000, 32000, 20),
+                                          (4, 32001, 32005, 32), (2, 4099, 4101, 1), (2, 262144, 262144, 20),
+                                          (130, 5000, 5000, 5)])
+def test_topm_bit_exact(N, V, stride, m):
+    rng = np.random.default_rng(V + m)
+    x = rng.standard_normal((N, stride)).astype(np.float32)
+    x[:, ::7] = np.round(x[:, ::7])                            # exact ties, also across chunk borders
+    x[:, V:] = 1e9                                             # padding beyond the vocabulary is never read
+    rv, ri = oracle.topm(x, m, vocab=V)
+    for _ in range(2):                                         # twice: the arrival counters must come back to zero
+        gv, gi, _ = H.run_topm(x, m, vocab=V)
+        np.testing.assert_array_equal(gi, ri)
+        np.testing.assert_array_equal(gv, rv)
+
+
+def test_topm_ties_nan_inf_and_argmax_agreement():
+    rng = np.random.default_rng(77)
+    x = rng.standard_normal((6, 9000)).astype(np.float32)
+    x[0, :] = 2.5                                              # all equal: indices 0..m-1
+    x[1, 100:140] = np.nan
+    x[1, 5000] = np.inf
+    x[2, :] = -np.inf
+    x[2, 8999] = np.nan                                        # counts as -inf: still indices 0..m-1
+    x[3, 17] = 0.0
+    x[3, 4] = -0.0
+    x[3, :] = np.where(x[3] > 0, -x[3], x[3])                  # zeros are the maxima: index 4 (the -0) before 17
+    x[3, 4], x[3, 17] = -0.0, 0.0
+    x[4, 4095], x[4, 4096] = 50.0, 50.0                        # a tie across the chunk border
+    rv, ri = oracle.topm(x, 20)
+    gv, gi, _ = H.run_topm(x, 20)
+    np.testing.assert_array_equal(gi, ri)
+    np.testing.assert_array_equal(gv, rv)
+    assert gi[0].tolist() == list(range(20)) and gi[2].tolist() == list(range(20))
+    assert gi[3, :2].tolist() == [4, 17] and gi[4, :2].tolist() == [4095, 4096] and gi[1, 0] == 5000
+    np.testing.assert_array_equal(H.run_topm(x, 1)[1][:, 0], oracle.argmax(x))
+
+
+def test_topm_rejects_bad_arguments_without_launching():
+    x = np.zeros((2, 64), np.float32)
+    ld = torch.from_numpy(x).cuda()
+    val = torch.full((2, 40), 3.0, dtype=torch.float32, device="cuda")
+    idx = torch.full((2, 40), -7, dtype=torch.int32, device="cuda")
+    for m, vocab in ((0, 64), (11, 10), (33, 64), (1, 0)):     # m < 1, m > vocab, m > FALCON_TOPM_MAX, empty rows
+        rc = H.ctx().falcon_topm(binding.topm_args(2, vocab, ld, 64, m, val, idx), check=False)
+        assert rc == binding.ERR_INVALID_ARG
+    rc = H.ctx().falcon_topm(binding.topm_args(2, 64, ld, 32, 4, val, idx), check=False)   # stride < vocab
+    assert rc == binding.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert (idx.cpu().numpy() == -7).all() and (val.cpu().numpy() == 3.0).all()
+
+
 # ------------------------------------------------------------------------ ABI
 def test_abi_rejects_bad_arguments_without_launching():
     rng = np.random.default_rng(1)
