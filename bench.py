@@ -179,6 +179,39 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def time_topm(ctx, binding, torch, dev, stream, logits_h, peak, m=20, copies=20, reps=20):
+    """falcon_topm (m = 20, Appendix A) on the step's logits shape: `copies` distinct matrices (more than L2)
+    in one CUDA graph, replayed; CUDA events on the launching stream.  Not part of the step."""
+    N, V = logits_h.shape
+    src = torch.from_numpy(logits_h).to(dev)
+    mats = [src.clone() for _ in range(copies)]
+    val = torch.empty((N, m), dtype=torch.float32, device=dev)
+    idx = torch.empty((N, m), dtype=torch.int32, device=dev)
+    calls = [binding.topm_args(N, V, x, V, m, val, idx) for x in mats]
+    with torch.cuda.stream(stream):
+        for a in calls:
+            ctx.falcon_topm(a)              # the first call allocates scratch: before the capture
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for a in calls:
+                ctx.falcon_topm(a)
+        for _ in range(3):
+            g.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        e1.record(stream)
+        stream.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (reps * copies)
+    nbytes = 4 * N * V + 8 * N * m
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"rows": N, "vocab": V, "m": m, "us_per_call": us, "bytes_per_call": nbytes,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                         "traffic": None}}
+
+
 # --------------------------------------------------------------------------- GPU arm
 def run_falcon(args):
     import torch
@@ -354,6 +387,9 @@ def run_falcon(args):
             dist.destroy_process_group()
         return
 
+    # ---------------- outside the step: the selection that grows the tree (the row next to the hot path) ----
+    topm = time_topm(ctx, binding, torch, dev, stream, logits_h, peak) if world == 1 else None
+
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         sl = oracle_sample_layers(spec, tb)
@@ -380,6 +416,7 @@ def run_falcon(args):
         "gpu_launches": args.steps * (NL + 2),
         "clocks": clocks,
         "cpu_baseline": cpu,
+        "extras": {"falcon_topm": topm},
         "wall_s_timed": t_wall,
     }
     print(json.dumps(line))
