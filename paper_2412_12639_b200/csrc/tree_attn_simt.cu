@@ -341,8 +341,8 @@ int launch_tree_attn_simt(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream
   const int n_tiles = (max_keys + kTileKeys - 1) / kTileKeys;
   if (splits == 0) {
     splits = (2 * ctx->sm_count + B * Hq - 1) / (B * Hq);
-    const int cap = n_tiles / 8 > 0 ? n_tiles / 8 : 1;  // at least 256 keys per split
-    if (splits > cap) splits = cap;
+    // down to one 32-key tile per split: a tile costs this kernel several microseconds (measured),
+    // far more than the merge of one more partial result
   }
   if (splits > 64) splits = 64;
   if (splits > n_tiles) splits = n_tiles;
