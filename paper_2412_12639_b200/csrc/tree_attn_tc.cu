@@ -10,19 +10,19 @@
 // touches global memory.
 //
 // Inside a CTA (320 threads):
-//   warp 8    TMA producer: the Q tile first, then K and V tiles (bf16, 128-byte swizzle) into a
+//   warp 0    TMA producer: the Q tile first, then K and V tiles (bf16, 128-byte swizzle) into a
 //             4-stage ring, completion on mbarriers; the first loads are issued by several warps.
-//   warp 9    one elected lane issues tcgen05.mma (the whole warp runs the loop).
+//   warp 1    one elected lane issues tcgen05.mma (the whole warp runs the loop).
 //             S = Q.K^T (M=128, N=64, K=128) reads Q and the K tile from shared memory;
 //             O += P.V (M=128, N=128, K=64) reads P from TMEM and the V tile from shared memory.
 //             tcgen05.commit signals the consumers.
-//   warps 0-7 softmax, one thread per (query row, stream or copy): per tile tcgen05.ld of the
+//   warps 2-9 softmax, one thread per (query row, stream or copy): per tile tcgen05.ld of the
 //             score row, tree mask from the node's ancestor bit set, online softmax with a lazily
 //             updated maximum (the accumulator is rescaled only when a weight would exceed 2^8),
 //             P written back to TMEM as packed bf16.  Units of more than 64 rows run two streams
-//             (warps 0-3 the even tiles, 4-7 the odd ones, one accumulator each, folded at the
+//             (warps 2-5 the even tiles, 6-9 the odd ones, one accumulator each, folded at the
 //             end); units of at most 64 rows hold the rows twice (lanes 0-63 and 64-127) and give
-//             each copy half of every tile's key columns (warps 0-3 only).
+//             each copy half of every tile's key columns (warps 2-5 only).
 // The partial rows cross the cluster as bf16 columns plus fp32 (max, sum).  All three falcon
 // kernels are launched programmatically dependent: set-up that touches no global memory runs
 // before griddepcontrol.wait and overlaps the previous kernel's drain.
@@ -51,9 +51,13 @@ constexpr int kStages = 4;         // ring depth: what shared memory leaves room
 // arrives together (the memory system serves the whole GPU's requests fairly), so a deep burst only
 // delays the first tile; the ring still lets the producer run ahead once tiles are consumed.
 constexpr int kPrefetch = 2;
-constexpr int kTcThreads = 320;    // warps 0-7 softmax (TMEM quadrant = warp % 4, stream = warp / 4), 8 producer, 9 MMA
-constexpr int kWarpProducer = 8;
-constexpr int kWarpMma = 9;
+// Warp roles.  A CTA's warps start one after the other (the tenth about 800 cycles after the first),
+// so the two warps with the longest set-up come first: 0 producer, 1 MMA, 2-9 softmax (TMEM
+// quadrant = warp % 4, stream = (warp - 2) / 4).
+constexpr int kTcThreads = 320;
+constexpr int kWarpProducer = 0;
+constexpr int kWarpMma = 1;
+constexpr int kWarpSm0 = 2;
 constexpr int kMaxSplits = 8;
 constexpr int kHostSeqs = 8;
 constexpr uint32_t kSpinLimit = 1u << 18;
@@ -367,7 +371,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   constexpr int kCols = kDup ? 32 : 64;  // key columns of a tile that one softmax thread handles
   constexpr int kGroups = kDup ? 2 : 1;  // partial results per row and CTA
-  // Softmax streams: with two, warps 0-3 take the even tiles of the CTA's run and warps 4-7 the odd
+  // Softmax streams: with two, warps 2-5 take the even tiles of the CTA's run and warps 6-9 the odd
   // ones, each stream with its own maximum, sum and accumulator.  Warps w and w+4 sit on the same
   // scheduler and reach the same TMEM lanes, so one stream's exponentials fill the gaps of the
   // other's loads, stores and barrier traffic, and after the loop the two threads of a row fold
@@ -381,9 +385,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int lane_row = q4 * 32 + lane;                       // TMEM lane, and the staging slot of its partial row
   const int grp = kDup ? (q4 >> 1) : 0;                      // which half of a tile's key columns
   const int row = kDup ? (q4 & 1) * 32 + lane : lane_row;    // query row of the tile
-  const bool is_sm = warp < 4 * kStreams;
-  const bool is_ld = warp < 4;                               // warps that issue one of the first loads
-  const int strm = kStreams == 2 ? ((warp >> 2) & 1) : 0;
+  const bool is_sm = warp >= kWarpSm0 && warp < kWarpSm0 + 4 * kStreams;
+  const int ld_slot = warp - kWarpSm0;                       // warps 2-5 issue one of the first loads each
+  const bool is_ld = ld_slot >= 0 && ld_slot < 4;
+  const int strm = kStreams == 2 ? (((warp - kWarpSm0) >> 2) & 1) : 0;
   const bool valid = is_sm && row < n_valid;
   const bool warp_valid = is_sm && (row - lane) < n_valid;
 
@@ -402,7 +407,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   // First loads, issued by several warps at once (a TMA instruction costs its issuing thread about
   // a hundred cycles): the producer takes the Q tile, in front so that it is not queued behind K/V,
-  // and the last stage; lane 0 of warps 0-3 takes stages 0-3.
+  // and the last stage; lane 0 of warps 2-5 takes stages 0-3.
   {
     const int pre = min(n_my, kPrefetch);
     if (lane == 0 && (is_ld || warp == kWarpProducer)) {
@@ -427,13 +432,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (split == 0 && mtile == 0 && kvh == 0 && (L + T > p.s_cap || T_real > FALCON_T_MAX))
           dev_status_or(p.status, b, FALCON_DEV_CAPACITY);
       }
-      if (kDup && n_my > 0 && (warp == 2 || warp == 3)) {  // the second copy of the Q tile, 64 rows further down
-        const int h = warp - 2;
+      if (kDup && n_my > 0 && (ld_slot == 2 || ld_slot == 3)) {  // the second copy of the Q tile, 64 rows further down
+        const int h = ld_slot - 2;
         tma_load_5d(smem_base + kOffQ + h * p.q_half_bytes + 64 * 128, &tm_q, bar(kBarQ), 0, 0, kvh,
                     node_base + mtile * (kBM / G), h);
       }
-      // warps 0-3: one stage each; the producer: whatever is left
-      for (int j = is_ld ? warp : 4; j < pre; j += is_ld ? 8 : 1) {
+      // warps 2-5: one stage each; the producer: whatever is left
+      for (int j = is_ld ? ld_slot : 4; j < pre; j += is_ld ? 8 : 1) {
         const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
         mbar_expect_tx(bar(kBarKVFull + j), 2 * kTileBytes);
         load_kv_tile(kdst, &tm_k, bar(kBarKVFull + j), key_begin + j * kBN, kvh, b);
