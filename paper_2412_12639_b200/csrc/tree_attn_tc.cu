@@ -251,7 +251,9 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+// Phase-1 arrival: orders nothing itself (the barrier initialisation it announces was released to the
+// cluster by fence.mbarrier_init), so it does not wait for this thread's loads in flight.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
 // Arrival that orders nothing: used where the barrier only keeps CTAs alive, so that it does not
 // have to wait for this thread's outstanding global stores.
 __device__ __forceinline__ void cluster_arrive_relaxed() {
@@ -386,8 +388,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int grp = kDup ? (q4 >> 1) : 0;                      // which half of a tile's key columns
   const int row = kDup ? (q4 & 1) * 32 + lane : lane_row;    // query row of the tile
   const bool is_sm = warp >= kWarpSm0 && warp < kWarpSm0 + 4 * kStreams;
-  const int ld_slot = warp - kWarpSm0;                       // warps 2-5 issue one of the first loads each
-  const bool is_ld = ld_slot >= 0 && ld_slot < 4;
   const int strm = kStreams == 2 ? (((warp - kWarpSm0) >> 2) & 1) : 0;
   const bool valid = is_sm && row < n_valid;
   const bool warp_valid = is_sm && (row - lane) < n_valid;
@@ -396,6 +396,43 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     FALCON_TRACE(lane == 0, 1);
     if (lane == kBarPFull || lane == kBarPFull + 1) mbar_init(bar(lane), n_sm_warps);  // one arrival per softmax warp
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncwarp();
+    // First loads, by this warp alone and before the CTA-wide barrier below (the CTA's last warps
+    // start hundreds of cycles after this one): the barriers they land on were initialised by this
+    // warp's own lanes.  Q goes first so that it is not queued behind K/V.
+    if (lane == 0) {
+      if (n_splits > 1) {
+        // this CTA will receive rows_mine rows of every other CTA's partial results
+        const int r0 = split * rows_per;
+        const int mine = max(0, min(n_valid, r0 + rows_per) - r0);
+        mbar_expect_tx(bar(kBarMrg), static_cast<uint32_t>((n_vs - kGroups) * mine) * kMrgRowBytes);
+      }
+      if (n_my > 0) {
+        const int node0 = node_base + mtile * (kBM / G);
+        if (kDup) {  // one load per 64-column half and copy (the second copy 64 rows further down)
+          mbar_expect_tx(bar(kBarQ), 4 * p.q_box_bytes);
+#pragma unroll
+          for (int c = 0; c < 2; ++c)
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+              tma_load_5d(smem_base + kOffQ + h * p.q_half_bytes + c * 64 * 128, &tm_q, bar(kBarQ), 0, 0, kvh, node0, h);
+        } else {
+          mbar_expect_tx(bar(kBarQ), p.q_box_bytes);
+          tma_load_5d(smem_base + kOffQ, &tm_q, bar(kBarQ), 0, 0, kvh, node0, 0);
+        }
+      }
+      const int pre = min(n_my, kPrefetch);
+      for (int j = 0; j < pre; ++j) {
+        const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
+        mbar_expect_tx(bar(kBarKVFull + j), 2 * kTileBytes);
+        load_kv_tile(kdst, &tm_k, bar(kBarKVFull + j), key_begin + j * kBN, kvh, b);
+        load_kv_tile(kdst + kTileBytes, &tm_v, bar(kBarKVFull + j), key_begin + j * kBN, kvh, b);
+      }
+      if (split == 0 && mtile == 0 && kvh == 0 && (L + T > p.s_cap || T_real > FALCON_T_MAX))
+        dev_status_or(p.status, b, FALCON_DEV_CAPACITY);
+      FALCON_TRACE(true, 2);
+    }
+    __syncwarp();
   }
   tc_fence_before();
   __syncthreads();
@@ -404,50 +441,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   FALCON_TRACE(tid == 0, 4);
   // Cluster phase 1: "my merge barrier exists".  Arrive now, wait just before the first remote copy.
   if (merge) cluster_arrive();
-
-  // First loads, issued by several warps at once (a TMA instruction costs its issuing thread about
-  // a hundred cycles): the producer takes the Q tile, in front so that it is not queued behind K/V,
-  // and the last stage; lane 0 of warps 2-5 takes stages 0-3.
-  {
-    const int pre = min(n_my, kPrefetch);
-    if (lane == 0 && (is_ld || warp == kWarpProducer)) {
-      if (warp == kWarpProducer) {
-        if (n_splits > 1) {
-          // this CTA will receive rows_mine rows of every other CTA's partial results
-          const int r0 = split * rows_per;
-          const int mine = max(0, min(n_valid, r0 + rows_per) - r0);
-          mbar_expect_tx(bar(kBarMrg), static_cast<uint32_t>((n_vs - kGroups) * mine) * kMrgRowBytes);
-        }
-        if (n_my > 0) {
-          const int node0 = node_base + mtile * (kBM / G);
-          if (kDup) {  // one load per 64-column half and copy; this thread takes the first copy
-            mbar_expect_tx(bar(kBarQ), 4 * p.q_box_bytes);
-            tma_load_5d(smem_base + kOffQ, &tm_q, bar(kBarQ), 0, 0, kvh, node0, 0);
-            tma_load_5d(smem_base + kOffQ + p.q_half_bytes, &tm_q, bar(kBarQ), 0, 0, kvh, node0, 1);
-          } else {
-            mbar_expect_tx(bar(kBarQ), p.q_box_bytes);
-            tma_load_5d(smem_base + kOffQ, &tm_q, bar(kBarQ), 0, 0, kvh, node0, 0);
-          }
-        }
-        if (split == 0 && mtile == 0 && kvh == 0 && (L + T > p.s_cap || T_real > FALCON_T_MAX))
-          dev_status_or(p.status, b, FALCON_DEV_CAPACITY);
-      }
-      if (kDup && n_my > 0 && (ld_slot == 2 || ld_slot == 3)) {  // the second copy of the Q tile, 64 rows further down
-        const int h = ld_slot - 2;
-        tma_load_5d(smem_base + kOffQ + h * p.q_half_bytes + 64 * 128, &tm_q, bar(kBarQ), 0, 0, kvh,
-                    node_base + mtile * (kBM / G), h);
-      }
-      // warps 2-5: one stage each; the producer: whatever is left
-      for (int j = is_ld ? ld_slot : 4; j < pre; j += is_ld ? 8 : 1) {
-        const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
-        mbar_expect_tx(bar(kBarKVFull + j), 2 * kTileBytes);
-        load_kv_tile(kdst, &tm_k, bar(kBarKVFull + j), key_begin + j * kBN, kvh, b);
-        load_kv_tile(kdst + kTileBytes, &tm_v, bar(kBarKVFull + j), key_begin + j * kBN, kvh, b);
-      }
-    }
-    __syncwarp();
-    FALCON_TRACE(warp == kWarpProducer && lane == 0, 2);
-  }
 
   if (warp == kWarpProducer) {
     // ================================ TMA producer (ring refills) ================================
