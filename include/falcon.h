@@ -110,8 +110,22 @@ typedef struct {
  * kernel      FALCON_ATTN_AUTO picks; the others force one kernel (tests).
  * n_splits    0 = automatic; else the number of KV splits per head (1..8 for
  *             the tensor-core kernel, 1..64 for the SIMT kernel).
+ * k/v_cache_next  optional hint (both or neither): the caches that the NEXT
+ *             falcon_tree_attn call on this stream will read (the following layer),
+ *             same shape and strides as k/v_cache.  When a layer's K/V is at most
+ *             48 MB, the tensor-core kernel asks the L2 cache to fetch their rows
+ *             [0, L_b + T_b) once its own loads are done, so that the fetch overlaps
+ *             this call's merge and the next call's set-up.  Nothing is read or
+ *             written through them by this call; results do not depend on the hint.
+ * flags       FALCON_ATTN_PREFIX_STABLE: the caller states that rows [0, L_b) of
+ *             k/v_cache were last written before the kernel that PRECEDES this call
+ *             on the stream started (true for a prefix written in an earlier step).
+ *             The tensor-core kernel may then request prefix tiles while that
+ *             preceding kernel is still finishing.  Needs the tree's host copies.
+ *             Without the flag every read waits for all earlier work of the stream.
  * ------------------------------------------------------------------------- */
 enum { FALCON_ATTN_AUTO = 0, FALCON_ATTN_SIMT = 1, FALCON_ATTN_TC = 2 };
+enum { FALCON_ATTN_PREFIX_STABLE = 1 };
 
 typedef struct {
   falcon_tree_desc tree;
@@ -128,6 +142,9 @@ typedef struct {
   const uint64_t* tree_mask;               /* optional [N][2]: bit t of row i = node i sees tree key t */
   int32_t kernel;
   int32_t n_splits;
+  const void* k_cache_next;                /* optional hint, see above                   */
+  const void* v_cache_next;
+  int32_t flags;                           /* FALCON_ATTN_* flag bits, 0 = none          */
 } falcon_attn_args;
 
 int falcon_tree_attn(falcon_ctx* ctx, const falcon_attn_args* args, void* stream);

@@ -62,6 +62,7 @@ constexpr int kMaxSplits = 8;
 constexpr int kHostSeqs = 8;
 constexpr uint32_t kSpinLimit = 1u << 18;
 constexpr uint32_t kSuspendHintNs = 2000;  // a waiting thread may sleep this long per try (it wakes when the phase completes)
+constexpr int64_t kNextPrefetchMaxBytes = 48ll << 20;  // a layer's K/V above this is not prefetched for the next call
 constexpr float kRescaleLimit = 256.f;  // largest weight tolerated before the row maximum is refreshed
 
 constexpr uint32_t kTileBytes = kBN * kD * 2;      // 16 KB: two 64-column halves of 8 KB
@@ -117,6 +118,8 @@ struct TcParams {
   // Per-sequence scalars from the caller's host copies (batches of up to kHostSeqs sequences):
   // with them the first loads do not have to wait for a round trip to global memory.
   int32_t have_host;
+  int32_t early_prefix;  // prefix tiles may be requested before the previous kernel has completed
+  int32_t prefetch_next;  // the next call's caches are known: fetch their rows into L2 at the end
   int32_t h_node_off[kHostSeqs + 1];
   int32_t h_prefix[kHostSeqs];
 };
@@ -174,6 +177,12 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map
 // One K or V tile: 64 keys x (2 halves of 64 head-dim columns), landing as two 128-byte-swizzled half tiles.
 __device__ __forceinline__ void load_kv_tile(uint32_t dst, const CUtensorMap* map, uint32_t bar, int k0, int kvh, int b) {
   tma_load_5d(dst, map, bar, 0, k0, 0, kvh, b);
+}
+// Hint: bring one K or V tile into L2 (nothing waits for it, nothing lands in shared memory).
+__device__ __forceinline__ void prefetch_kv_tile_l2(const CUtensorMap* map, int k0, int kvh, int b) {
+  asm volatile("cp.async.bulk.prefetch.tensor.5d.L2.global.tile [%0, {%1, %2, %3, %4, %5}];" ::"l"(map), "r"(0), "r"(k0),
+               "r"(0), "r"(kvh), "r"(b)
+               : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -295,7 +304,8 @@ __device__ __forceinline__ uint64_t window64(uint64_t lo, uint64_t hi, int off) 
 template <bool kDup>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                    const __grid_constant__ CUtensorMap tm_v, const TcParams p) {
+                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k_next,
+                    const __grid_constant__ CUtensorMap tm_v_next, const TcParams p) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t s_bars[kNumBars];
   __shared__ uint32_t s_tmem_base;
@@ -327,17 +337,41 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  int node_base = 0, T_real = 0, L_raw = 0;
+  int n_early = 0;  // K/V tiles requested before the wait below
+  if (p.have_host) {
+    node_base = p.h_node_off[b];
+    T_real = p.h_node_off[b + 1] - node_base;
+    L_raw = p.h_prefix[b];
+    // Prefix rows that the caller declares stable (written before the kernel that precedes this one
+    // in the stream started) may be requested while that kernel is still finishing.
+    if (p.early_prefix && warp == kWarpProducer) {
+      __syncwarp();
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      if (lane == 0 && mtile * kBM < min(T_real, FALCON_T_MAX) * G) {
+        const int Tq = min(T_real, FALCON_T_MAX), Lq = min(max(L_raw, 0), p.s_cap);
+        const int Sv = min(max(L_raw, 0) + Tq, p.s_cap);
+        const int nt = (Sv + kBN - 1) / kBN;
+        const int kb = min(Sv, ((split * nt) / n_splits) * kBN);
+        const int ke = min(Sv, (((split + 1) * nt) / n_splits) * kBN);
+        const int nm = (ke - kb + kBN - 1) / kBN;
+        for (int j = 0; j < min(nm, kPrefetch) && kb + (j + 1) * kBN <= Lq; ++j) {
+          const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
+          mbar_expect_tx(bar(kBarKVFull + j), 2 * kTileBytes);
+          load_kv_tile(kdst, &tm_k, bar(kBarKVFull + j), kb + j * kBN, kvh, b);
+          load_kv_tile(kdst + kTileBytes, &tm_v, bar(kBarKVFull + j), kb + j * kBN, kvh, b);
+          ++n_early;
+        }
+      }
+    }
+  }
   // Everything below may read what earlier kernels of the stream wrote (tree arrays, q, the tree's
   // K/V rows) and writes `out`: wait until they have completed.  Then let the next kernel's CTAs
   // be scheduled as this grid's CTAs leave their SMs (a no-op without programmatic launch).
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  int node_base, T_real, L_raw;
-  if (p.have_host) {
-    node_base = p.h_node_off[b];
-    T_real = p.h_node_off[b + 1] - node_base;
-    L_raw = p.h_prefix[b];
-  } else {
+  if (!p.have_host) {
     node_base = p.node_off[b];
     T_real = p.node_off[b + 1] - node_base;
     L_raw = p.prefix_len[b];
@@ -364,7 +398,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int key_end = min(S_valid, (((split + 1) * n_tiles) / n_splits) * kBN);
   const int n_my = (key_end - key_begin + kBN - 1) / kBN;
 
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   volatile int* abort_flag = &s_abort;
 
@@ -422,7 +455,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
       }
       const int pre = min(n_my, kPrefetch);
-      for (int j = 0; j < pre; ++j) {
+      for (int j = n_early; j < pre; ++j) {
         const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
         mbar_expect_tx(bar(kBarKVFull + j), 2 * kTileBytes);
         load_kv_tile(kdst, &tm_k, bar(kBarKVFull + j), key_begin + j * kBN, kvh, b);
@@ -462,6 +495,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         mbar_expect_tx(bar(kBarKVFull + st), 2 * kTileBytes);
         load_kv_tile(kdst, &tm_k, bar(kBarKVFull + st), k0, kvh, b);
         load_kv_tile(vdst, &tm_v, bar(kBarKVFull + st), k0, kvh, b);
+      }
+    }
+    // The caller named the caches of the call that follows on this stream: once this CTA's own last
+    // tile has landed, ask L2 for the same key range of those caches.  The fetch runs while this
+    // launch merges and the next one sets up, a time in which HBM would otherwise sit idle.
+    if (p.prefetch_next && mtile == 0 && n_my > 0) {
+      const int jl = n_my - 1;
+      bool ok = true;
+      if (lane == 0) ok = mbar_wait(bar(kBarKVFull + jl % kStages), (jl / kStages) & 1, abort_flag);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      for (int j = lane; ok && j < n_my; j += 32) {
+        prefetch_kv_tile_l2(&tm_k_next, key_begin + j * kBN, kvh, b);
+        prefetch_kv_tile_l2(&tm_v_next, key_begin + j * kBN, kvh, b);
       }
     }
   } else if (warp == kWarpMma) {
@@ -1064,6 +1110,22 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
     return FALCON_ERR_CUDA;
   }
   const CUtensorMap mq = *tq, mk = *tk, mv = *tv;  // copies: later cache growth must not move what we pass
+  // The next call's caches (same shape and strides), if the caller named them and a layer's K/V is
+  // small enough to wait in L2 next to this layer's.
+  CUtensorMap mkn = mk, mvn = mv;
+  bool prefetch_next = false;
+  if (a.k_cache_next && a.v_cache_next) {
+    const int64_t kv_bytes = static_cast<int64_t>(B) * Hkv * (a.tree.max_prefix_len + a.tree.max_tree) * kD * 2 * 2;
+    if (kv_bytes <= kNextPrefetchMaxBytes) {
+      const CUtensorMap* tkn = get_tmap(ctx, a.k_cache_next, kv_dims, kv_strides, kv_box);
+      const CUtensorMap* tvn = get_tmap(ctx, a.v_cache_next, kv_dims, kv_strides, kv_box);
+      if (tkn && tvn) {
+        mkn = *tkn;
+        mvn = *tvn;
+        prefetch_next = true;
+      }
+    }
+  }
 
   TcParams p;
   p.Hq = Hq;
@@ -1080,6 +1142,8 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   p.status = a.tree.status;
   p.tree_mask = a.tree_mask;
   p.have_host = 0;
+  p.early_prefix = (a.flags & FALCON_ATTN_PREFIX_STABLE) ? 1 : 0;
+  p.prefetch_next = prefetch_next ? 1 : 0;
   if (a.tree.prefix_len_host && a.tree.node_off_host && B <= kHostSeqs) {
     p.have_host = 1;
     for (int i = 0; i <= B; ++i) p.h_node_off[i] = a.tree.node_off_host[i];
@@ -1104,8 +1168,8 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  cudaError_t e = dup ? cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<true>, mq, mk, mv, p)
-                      : cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<false>, mq, mk, mv, p);
+  cudaError_t e = dup ? cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<true>, mq, mk, mv, mkn, mvn, p)
+                      : cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<false>, mq, mk, mv, mkn, mvn, p);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tree_attn_tc_kernel launch");
   return FALCON_OK;
 }
