@@ -285,11 +285,8 @@ def run_falcon(args):
     vptr = torch.tensor([cache[l, 1].data_ptr() for l in range(NL)], dtype=torch.int64, device=dev)
     strides = tuple(int(s) for s in cache[0, 0].stride()[:3])
 
-    # Every layer but the last names the next layer's caches (an L2 prefetch hint; the last layer's call is
-    # followed by the acceptance, not by another layer).  The prefix rows were written in earlier steps.
+    # the prefix rows were written in earlier steps: the kernel may ask for them while the previous launch drains
     attn = [binding.attn_args(tree, Hq, Hkv, D, scale, q_all[l], out_all[l], cache[l, 0], cache[l, 1], strides, s_cap,
-                              k_cache_next=cache[l + 1, 0] if l + 1 < NL else None,
-                              v_cache_next=cache[l + 1, 1] if l + 1 < NL else None,
                               flags=binding.ATTN_PREFIX_STABLE)
             for l in range(NL)]
     acc = binding.accept_args(tree, spec.vocab, logits, logits.shape[1], g, path, 128, n_path, nxt)

@@ -110,13 +110,6 @@ typedef struct {
  * kernel      FALCON_ATTN_AUTO picks; the others force one kernel (tests).
  * n_splits    0 = automatic; else the number of KV splits per head (1..8 for
  *             the tensor-core kernel, 1..64 for the SIMT kernel).
- * k/v_cache_next  optional hint (both or neither): the caches that the NEXT
- *             falcon_tree_attn call on this stream will read (the following layer),
- *             same shape and strides as k/v_cache.  When a layer's K/V is at most
- *             48 MB, the tensor-core kernel asks the L2 cache to fetch their rows
- *             [0, L_b + T_b) once its own loads are done, so that the fetch overlaps
- *             this call's merge and the next call's set-up.  Nothing is read or
- *             written through them by this call; results do not depend on the hint.
  * flags       FALCON_ATTN_PREFIX_STABLE: the caller states that rows [0, L_b) of
  *             k/v_cache were last written before the kernel that PRECEDES this call
  *             on the stream started (true for a prefix written in an earlier step).
@@ -142,8 +135,6 @@ typedef struct {
   const uint64_t* tree_mask;               /* optional [N][2]: bit t of row i = node i sees tree key t */
   int32_t kernel;
   int32_t n_splits;
-  const void* k_cache_next;                /* optional hint, see above                   */
-  const void* v_cache_next;
   int32_t flags;                           /* FALCON_ATTN_* flag bits, 0 = none          */
 } falcon_attn_args;
 

@@ -62,7 +62,6 @@ constexpr int kMaxSplits = 8;
 constexpr int kHostSeqs = 8;
 constexpr uint32_t kSpinLimit = 1u << 18;
 constexpr uint32_t kSuspendHintNs = 2000;  // a waiting thread may sleep this long per try (it wakes when the phase completes)
-constexpr int64_t kNextPrefetchMaxBytes = 48ll << 20;  // a layer's K/V above this is not prefetched for the next call
 constexpr float kRescaleLimit = 256.f;  // largest weight tolerated before the row maximum is refreshed
 
 constexpr uint32_t kTileBytes = kBN * kD * 2;      // 16 KB: two 64-column halves of 8 KB
@@ -119,7 +118,6 @@ struct TcParams {
   // with them the first loads do not have to wait for a round trip to global memory.
   int32_t have_host;
   int32_t early_prefix;  // prefix tiles may be requested before the previous kernel has completed
-  int32_t prefetch_next;  // the next call's caches are known: fetch their rows into L2 at the end
   int32_t h_node_off[kHostSeqs + 1];
   int32_t h_prefix[kHostSeqs];
 };
@@ -177,12 +175,6 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map
 // One K or V tile: 64 keys x (2 halves of 64 head-dim columns), landing as two 128-byte-swizzled half tiles.
 __device__ __forceinline__ void load_kv_tile(uint32_t dst, const CUtensorMap* map, uint32_t bar, int k0, int kvh, int b) {
   tma_load_5d(dst, map, bar, 0, k0, 0, kvh, b);
-}
-// Hint: bring one K or V tile into L2 (nothing waits for it, nothing lands in shared memory).
-__device__ __forceinline__ void prefetch_kv_tile_l2(const CUtensorMap* map, int k0, int kvh, int b) {
-  asm volatile("cp.async.bulk.prefetch.tensor.5d.L2.global.tile [%0, {%1, %2, %3, %4, %5}];" ::"l"(map), "r"(0), "r"(k0),
-               "r"(0), "r"(kvh), "r"(b)
-               : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -304,8 +296,7 @@ __device__ __forceinline__ uint64_t window64(uint64_t lo, uint64_t hi, int off) 
 template <bool kDup>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k_next,
-                    const __grid_constant__ CUtensorMap tm_v_next, const TcParams p) {
+                    const __grid_constant__ CUtensorMap tm_v, const TcParams p) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t s_bars[kNumBars];
   __shared__ uint32_t s_tmem_base;
@@ -495,19 +486,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         mbar_expect_tx(bar(kBarKVFull + st), 2 * kTileBytes);
         load_kv_tile(kdst, &tm_k, bar(kBarKVFull + st), k0, kvh, b);
         load_kv_tile(vdst, &tm_v, bar(kBarKVFull + st), k0, kvh, b);
-      }
-    }
-    // The caller named the caches of the call that follows on this stream: once this CTA's own last
-    // tile has landed, ask L2 for the same key range of those caches.  The fetch runs while this
-    // launch merges and the next one sets up, a time in which HBM would otherwise sit idle.
-    if (p.prefetch_next && mtile == 0 && n_my > 0) {
-      const int jl = n_my - 1;
-      bool ok = true;
-      if (lane == 0) ok = mbar_wait(bar(kBarKVFull + jl % kStages), (jl / kStages) & 1, abort_flag);
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      for (int j = lane; ok && j < n_my; j += 32) {
-        prefetch_kv_tile_l2(&tm_k_next, key_begin + j * kBN, kvh, b);
-        prefetch_kv_tile_l2(&tm_v_next, key_begin + j * kBN, kvh, b);
       }
     }
   } else if (warp == kWarpMma) {
@@ -1110,23 +1088,6 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
     return FALCON_ERR_CUDA;
   }
   const CUtensorMap mq = *tq, mk = *tk, mv = *tv;  // copies: later cache growth must not move what we pass
-  // The next call's caches (same shape and strides), if the caller named them and a layer's K/V is
-  // small enough to wait in L2 next to this layer's.
-  CUtensorMap mkn = mk, mvn = mv;
-  bool prefetch_next = false;
-  if (a.k_cache_next && a.v_cache_next) {
-    const int64_t kv_bytes = static_cast<int64_t>(B) * Hkv * (a.tree.max_prefix_len + a.tree.max_tree) * kD * 2 * 2;
-    if (kv_bytes <= kNextPrefetchMaxBytes) {
-      const CUtensorMap* tkn = get_tmap(ctx, a.k_cache_next, kv_dims, kv_strides, kv_box);
-      const CUtensorMap* tvn = get_tmap(ctx, a.v_cache_next, kv_dims, kv_strides, kv_box);
-      if (tkn && tvn) {
-        mkn = *tkn;
-        mvn = *tvn;
-        prefetch_next = true;
-      }
-    }
-  }
-
   TcParams p;
   p.Hq = Hq;
   p.Hkv = Hkv;
@@ -1143,7 +1104,6 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   p.tree_mask = a.tree_mask;
   p.have_host = 0;
   p.early_prefix = (a.flags & FALCON_ATTN_PREFIX_STABLE) ? 1 : 0;
-  p.prefetch_next = prefetch_next ? 1 : 0;
   if (a.tree.prefix_len_host && a.tree.node_off_host && B <= kHostSeqs) {
     p.have_host = 1;
     for (int i = 0; i <= B; ++i) p.h_node_off[i] = a.tree.node_off_host[i];
@@ -1168,8 +1128,8 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  cudaError_t e = dup ? cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<true>, mq, mk, mv, mkn, mvn, p)
-                      : cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<false>, mq, mk, mv, mkn, mvn, p);
+  cudaError_t e = dup ? cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<true>, mq, mk, mv, p)
+                      : cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<false>, mq, mk, mv, p);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tree_attn_tc_kernel launch");
   return FALCON_OK;
 }

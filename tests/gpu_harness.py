@@ -66,9 +66,8 @@ def make_trees(sizes, prefs, rng, vocab=100, parents=None) -> synth.TreeBatch:
 
 
 def run_attn(dt: DevTrees, Hq, Hkv, D, q, k, v, s_cap=None, scale=None, kernel=binding.ATTN_AUTO, n_splits=0,
-             k_tree=None, v_tree=None, tree_mask=None, check=True, host_copies=False, flags=0, next_kv=None):
-    """q [N,Hq,D], k/v [B,Hkv,s_cap,D] uint16 bit patterns -> (out bits [N,Hq,D], rc).
-    next_kv: (k, v) bit patterns of the caches named as the next call's (prefetch hint)."""
+             k_tree=None, v_tree=None, tree_mask=None, check=True, host_copies=False, flags=0):
+    """q [N,Hq,D], k/v [B,Hkv,s_cap,D] uint16 bit patterns -> (out bits [N,Hq,D], rc)."""
     scale = 1.0 / math.sqrt(D) if scale is None else scale
     qd, kd, vd = dev_bf16(q), dev_bf16(k), dev_bf16(v)
     out = torch.full_like(qd, float("nan"))
@@ -76,10 +75,9 @@ def run_attn(dt: DevTrees, Hq, Hkv, D, q, k, v, s_cap=None, scale=None, kernel=b
     vtd = dev_bf16(v_tree) if v_tree is not None else None
     md = torch.from_numpy(np.ascontiguousarray(tree_mask).view(np.int64)).cuda() if tree_mask is not None else None
     strides = tuple(int(s) for s in kd.stride()[:3])
-    knd, vnd = (dev_bf16(next_kv[0]), dev_bf16(next_kv[1])) if next_kv is not None else (None, None)
     a = binding.attn_args(dt.desc(host_copies=host_copies), Hq, Hkv, D, scale, qd, out, kd, vd, strides,
                           kd.shape[2] if s_cap is None else s_cap, k_tree=ktd, v_tree=vtd, tree_mask=md,
-                          kernel=kernel, n_splits=n_splits, k_cache_next=knd, v_cache_next=vnd, flags=flags)
+                          kernel=kernel, n_splits=n_splits, flags=flags)
     rc = ctx().falcon_tree_attn(a, check=check)
     torch.cuda.synchronize()
     return host_bits(out), rc
