@@ -344,8 +344,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int Tq = min(T_real, FALCON_T_MAX), Lq = min(max(L_raw, 0), p.s_cap);
         const int Sv = min(max(L_raw, 0) + Tq, p.s_cap);
         const int nt = (Sv + kBN - 1) / kBN;
-        const int kb = min(Sv, ((split * nt) / n_splits) * kBN);
-        const int ke = min(Sv, (((split + 1) * nt) / n_splits) * kBN);
+        const int kb = min(Sv, ((split * nt + n_splits - 1) / n_splits) * kBN);
+        const int ke = min(Sv, (((split + 1) * nt + n_splits - 1) / n_splits) * kBN);
         const int nm = (ke - kb + kBN - 1) / kBN;
         for (int j = 0; j < min(nm, kPrefetch) && kb + (j + 1) * kBN <= Lq; ++j) {
           const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
@@ -383,10 +383,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const int Lc = min(L, p.s_cap);
   const int S_valid = min(L + T, p.s_cap);  // keys that exist below the cache capacity
   // Whole tiles per split, as even as they go (an iteration costs about the same whatever part of
-  // its 64 keys is real, so fewer iterations beat equal key counts).
+  // its 64 keys is real, so fewer iterations beat equal key counts).  The boundaries are rounded
+  // up, so a longer run goes to an early split: the last one has the tree's tiles, whose masked
+  // softmax pass is the slowest, and should not be the cluster's straggler as well.
   const int n_tiles = (S_valid + kBN - 1) / kBN;
-  const int key_begin = min(S_valid, ((split * n_tiles) / n_splits) * kBN);
-  const int key_end = min(S_valid, (((split + 1) * n_tiles) / n_splits) * kBN);
+  const int key_begin = min(S_valid, ((split * n_tiles + n_splits - 1) / n_splits) * kBN);
+  const int key_end = min(S_valid, (((split + 1) * n_tiles + n_splits - 1) / n_splits) * kBN);
   const int n_my = (key_end - key_begin + kBN - 1) / kBN;
 
   unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
