@@ -111,8 +111,9 @@ typedef struct {
  * n_splits    0 = automatic; else the number of KV splits per head (1..8 for
  *             the tensor-core kernel, 1..64 for the SIMT kernel).
  * flags       FALCON_ATTN_PREFIX_STABLE: the caller states that rows [0, L_b) of
- *             k/v_cache were last written before the kernel that PRECEDES this call
- *             on the stream started (true for a prefix written in an earlier step).
+ *             k/v_cache were last written by work that had COMPLETED before the
+ *             kernel that precedes this call on the stream started (true for a
+ *             prefix written in an earlier decoding step).
  *             The tensor-core kernel may then request prefix tiles while that
  *             preceding kernel is still finishing.  Needs the tree's host copies.
  *             Without the flag every read waits for all earlier work of the stream.
