@@ -64,3 +64,34 @@ def test_binding_structs_match_header_field_order():
             for part in decl.split(","):
                 fields.append(re.findall(r"([A-Za-z_0-9]+)\s*$", part.strip())[0])
         assert fields == [f[0] for f in struct._fields_], cname
+
+
+def test_binding_structs_match_the_compiled_layout(tmp_path):
+    """The header compiles as plain C, and the size of every argument struct and the offset of every
+    field, as the C compiler lays them out, equal those of the ctypes structures."""
+    import shutil
+    import subprocess
+    from paper_2412_12639_b200 import binding
+    cc = shutil.which("gcc") or shutil.which("cc")
+    if cc is None:
+        pytest.skip("no C compiler")
+    structs = (("falcon_tree_desc", binding.TreeDesc), ("falcon_attn_args", binding.AttnArgs),
+               ("falcon_accept_args", binding.AcceptArgs), ("falcon_topm_args", binding.TopmArgs),
+               ("falcon_compact_args", binding.CompactArgs))
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "falcon.h"', 'int main(void) {']
+    for cname, st in structs:
+        lines.append('  printf("%s %%zu\\n", sizeof(%s));' % (cname, cname))
+        for fname, _ in st._fields_:
+            lines.append('  printf("%s.%s %%zu\\n", offsetof(%s, %s));' % (cname, fname, cname, fname))
+    lines += ['  return 0;', '}']
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run([cc, "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)],
+                   check=True)
+    got = dict(line.split() for line in subprocess.run([str(exe)], check=True, capture_output=True,
+                                                       text=True).stdout.splitlines())
+    for cname, st in structs:
+        assert int(got[cname]) == ctypes.sizeof(st), cname
+        for fname, _ in st._fields_:
+            assert int(got["%s.%s" % (cname, fname)]) == getattr(st, fname).offset, "%s.%s" % (cname, fname)
