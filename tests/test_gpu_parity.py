@@ -508,6 +508,37 @@ def test_attn_tc_stable_prefix_flag_changes_nothing(T, G, L, splits):
     assert not dt.status.cpu().numpy().any()
 
 
+def test_attn_tc_stable_prefix_back_to_back_launches_match_single_launches():
+    """Eight layers launched back to back on one stream with the stable-prefix flag (each launch asks for
+    its prefix tiles while the one before it is still finishing) give, bit for bit, what each layer gives
+    when launched alone without the flag."""
+    import torch
+    spec = synth.SPECS["v7b"]
+    tb = synth.make_trees(spec)
+    dt = H.DevTrees(tb)
+    Hq, Hkv, D = spec.n_q_heads, spec.n_kv_heads, spec.head_dim
+    layers = [synth.make_layer_qkv(spec, tb, l) for l in range(8)]
+    alone = []
+    for q, k, v in layers:
+        out, rc = H.run_attn(dt, Hq, Hkv, D, q, k, v, kernel=binding.ATTN_TC, check=False)
+        tc_or_skip(rc)
+        alone.append(out)
+    dev = [(H.dev_bf16(q), H.dev_bf16(k), H.dev_bf16(v)) for q, k, v in layers]
+    outs = [torch.full_like(q, float("nan")) for q, _, _ in dev]
+    tree = dt.desc(host_copies=True)
+    args = [binding.attn_args(tree, Hq, Hkv, D, 1.0 / np.sqrt(D), q, o, k, v, tuple(int(x) for x in k.stride()[:3]),
+                              k.shape[2], kernel=binding.ATTN_TC, flags=binding.ATTN_PREFIX_STABLE)
+            for (q, k, v), o in zip(dev, outs)]
+    torch.cuda.synchronize()
+    for _ in range(3):
+        for a in args:
+            H.ctx().falcon_tree_attn(a)
+    torch.cuda.synchronize()
+    for o, ref in zip(outs, alone):
+        np.testing.assert_array_equal(H.host_bits(o), ref)
+    assert not dt.status.cpu().numpy().any()
+
+
 @pytest.mark.parametrize("seed", range(6))
 def test_attn_tc_random_batches_and_splits(seed):
     """Random batches (ragged trees and prefixes around the tile edges), head groupings and forced
