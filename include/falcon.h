@@ -118,7 +118,7 @@ typedef struct {
  *             preceding kernel is still finishing.  Needs the tree's host copies.
  *             Without the flag every read waits for all earlier work of the stream.
  * ------------------------------------------------------------------------- */
-enum { FALCON_ATTN_AUTO = 0, FALCON_ATTN_SIMT = 1, FALCON_ATTN_TC = 2 };
+enum { FALCON_ATTN_AUTO = 0, FALCON_ATTN_SIMT = 1, FALCON_ATTN_TC = 2, FALCON_ATTN_TCK = 3 };
 enum { FALCON_ATTN_PREFIX_STABLE = 1 };
 
 typedef struct {

@@ -15,7 +15,7 @@ from typing import Optional
 T_MAX = 128
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_BAD_TREE, ERR_CAPACITY, ERR_TIMEOUT = range(7)
 DEV_BAD_TREE, DEV_CAPACITY, DEV_BAD_PATH, DEV_TIMEOUT = 1, 2, 4, 8
-ATTN_AUTO, ATTN_SIMT, ATTN_TC = 0, 1, 2
+ATTN_AUTO, ATTN_SIMT, ATTN_TC, ATTN_TCK = 0, 1, 2, 3
 ATTN_PREFIX_STABLE = 1
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libfalcon.so")

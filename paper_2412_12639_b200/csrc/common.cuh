@@ -21,8 +21,14 @@ struct falcon_ctx {
   int* tickets = nullptr;
   size_t n_tickets = 0;
   std::string last_error;
-  // Cached TMA descriptors (opaque here; owned by tree_attn_tc.cu).
+  // Cached TMA descriptors (opaque here; owned by tc_util.cuh).
   void* tmap_cache = nullptr;
+  // Per-context launch state of the tensor-core attention kernels: whether the dynamic shared
+  // memory limit has been raised on this device, and how many clusters of each size fit at once
+  // (0 = not asked yet, -1 = none).  Index 0: rows-on-lanes kernel; 1, 2: keys-on-lanes kernel
+  // (small and large query block).
+  bool attn_attr_set[3] = {false, false, false};
+  int attn_resident[3][9] = {};
 };
 
 namespace falcon {
@@ -39,6 +45,8 @@ int launch_tree_topm(falcon_ctx* ctx, const falcon_topm_args& a, cudaStream_t s)
 int launch_tree_attn_simt(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s);
 int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s);
 bool tree_attn_tc_supports(const falcon_ctx* ctx, const falcon_attn_args& a);
+int launch_tree_attn_tck(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s);
+bool tree_attn_tck_supports(const falcon_ctx* ctx, const falcon_attn_args& a);
 void tree_attn_tc_release(falcon_ctx* ctx);
 
 #ifdef __CUDACC__

@@ -131,8 +131,12 @@ int falcon_tree_attn(falcon_ctx* ctx, const falcon_attn_args* a, void* stream) {
     case FALCON_ATTN_TC:
       if (!tree_attn_tc_supports(ctx, *a)) return FALCON_ERR_UNSUPPORTED;
       return launch_tree_attn_tc(ctx, *a, s);
+    case FALCON_ATTN_TCK:
+      if (!tree_attn_tck_supports(ctx, *a)) return FALCON_ERR_UNSUPPORTED;
+      return launch_tree_attn_tck(ctx, *a, s);
     case FALCON_ATTN_AUTO:
       if (tree_attn_tc_supports(ctx, *a)) return launch_tree_attn_tc(ctx, *a, s);
+      if (tree_attn_tck_supports(ctx, *a)) return launch_tree_attn_tck(ctx, *a, s);
       return launch_tree_attn_simt(ctx, *a, s);
     default:
       return FALCON_ERR_INVALID_ARG;

@@ -14,7 +14,8 @@ import gpu_harness as H
 
 pytestmark = pytest.mark.gpu
 
-KERNELS = [binding.ATTN_SIMT, binding.ATTN_TC]
+KERNELS = [binding.ATTN_SIMT, binding.ATTN_TC, binding.ATTN_TCK]
+TC_KERNELS = [binding.ATTN_TC, binding.ATTN_TCK]      # queries / keys on the tensor-memory lanes
 
 
 def tc_or_skip(rc):
@@ -472,24 +473,26 @@ def test_compact_path_longer_than_the_declared_max_tree_is_refused():
     np.testing.assert_array_equal(gv[0][1, :, :8], ref_v[1, :, :8])
 
 
+@pytest.mark.parametrize("tck", TC_KERNELS)
 @pytest.mark.parametrize("T,G,L,splits", [(60, 1, 700, 1), (60, 1, 700, 4), (32, 2, 100, 2), (17, 1, 0, 1),
                                            (80, 1, 30, 2), (80, 1, 500, 1), (128, 1, 64, 3), (16, 8, 1000, 5)])
-def test_attn_tc_row_arrangements(T, G, L, splits):
+def test_attn_tc_row_arrangements(T, G, L, splits, tck):
     """Both arrangements of the tensor-core kernel (two copies of at most 64 rows; two streams on
     alternate tiles, including runs of a single tile where the second stream has nothing) at forced splits."""
     rng = np.random.default_rng(100 * T + 10 * G + splits)
     Hkv = 2
     tb, q, k, v = random_case(rng, [T], [L], Hkv * G, Hkv, 128, slack=1)
     ref = oracle_attn(tb, Hkv * G, Hkv, 128, q, k, v)
-    out, rc = H.run_attn(H.DevTrees(tb), Hkv * G, Hkv, 128, q, k, v, kernel=binding.ATTN_TC, n_splits=splits,
+    out, rc = H.run_attn(H.DevTrees(tb), Hkv * G, Hkv, 128, q, k, v, kernel=tck, n_splits=splits,
                          check=False)
     tc_or_skip(rc)
     H.assert_attn_close(out, ref, tb.node_off)
 
 
+@pytest.mark.parametrize("tck", TC_KERNELS)
 @pytest.mark.parametrize("T,G,L,splits", [(60, 1, 1024, 0), (60, 1, 700, 4), (80, 1, 500, 3), (16, 8, 1000, 5),
                                            (20, 1, 10, 2), (33, 2, 0, 1)])
-def test_attn_tc_stable_prefix_flag_changes_nothing(T, G, L, splits):
+def test_attn_tc_stable_prefix_flag_changes_nothing(T, G, L, splits, tck):
     """FALCON_ATTN_PREFIX_STABLE (prefix tiles requested before the preceding kernel has drained) leaves the
     output bit-identical, with the host copies it acts on and without them."""
     rng = np.random.default_rng(7000 + 100 * T + 10 * G + splits)
@@ -497,18 +500,19 @@ def test_attn_tc_stable_prefix_flag_changes_nothing(T, G, L, splits):
     tb, q, k, v = random_case(rng, [T, max(1, T // 2)], [L, L // 3], Hkv * G, Hkv, 128, slack=1)
     ref = oracle_attn(tb, Hkv * G, Hkv, 128, q, k, v)
     dt = H.DevTrees(tb)
-    base, rc = H.run_attn(dt, Hkv * G, Hkv, 128, q, k, v, kernel=binding.ATTN_TC, n_splits=splits, check=False,
+    base, rc = H.run_attn(dt, Hkv * G, Hkv, 128, q, k, v, kernel=tck, n_splits=splits, check=False,
                           host_copies=True)
     tc_or_skip(rc)
     H.assert_attn_close(base, ref, tb.node_off)
     for hc in (True, False):
-        out, _ = H.run_attn(dt, Hkv * G, Hkv, 128, q, k, v, kernel=binding.ATTN_TC, n_splits=splits,
+        out, _ = H.run_attn(dt, Hkv * G, Hkv, 128, q, k, v, kernel=tck, n_splits=splits,
                             host_copies=hc, flags=binding.ATTN_PREFIX_STABLE)
         np.testing.assert_array_equal(out, base)
     assert not dt.status.cpu().numpy().any()
 
 
-def test_attn_tc_stable_prefix_back_to_back_launches_match_single_launches():
+@pytest.mark.parametrize("tck", TC_KERNELS)
+def test_attn_tc_stable_prefix_back_to_back_launches_match_single_launches(tck):
     """Eight layers launched back to back on one stream with the stable-prefix flag (each launch asks for
     its prefix tiles while the one before it is still finishing) give, bit for bit, what each layer gives
     when launched alone without the flag."""
@@ -520,14 +524,14 @@ def test_attn_tc_stable_prefix_back_to_back_launches_match_single_launches():
     layers = [synth.make_layer_qkv(spec, tb, l) for l in range(8)]
     alone = []
     for q, k, v in layers:
-        out, rc = H.run_attn(dt, Hq, Hkv, D, q, k, v, kernel=binding.ATTN_TC, check=False)
+        out, rc = H.run_attn(dt, Hq, Hkv, D, q, k, v, kernel=tck, check=False)
         tc_or_skip(rc)
         alone.append(out)
     dev = [(H.dev_bf16(q), H.dev_bf16(k), H.dev_bf16(v)) for q, k, v in layers]
     outs = [torch.full_like(q, float("nan")) for q, _, _ in dev]
     tree = dt.desc(host_copies=True)
     args = [binding.attn_args(tree, Hq, Hkv, D, 1.0 / np.sqrt(D), q, o, k, v, tuple(int(x) for x in k.stride()[:3]),
-                              k.shape[2], kernel=binding.ATTN_TC, flags=binding.ATTN_PREFIX_STABLE)
+                              k.shape[2], kernel=tck, flags=binding.ATTN_PREFIX_STABLE)
             for (q, k, v), o in zip(dev, outs)]
     torch.cuda.synchronize()
     for _ in range(3):
@@ -539,8 +543,9 @@ def test_attn_tc_stable_prefix_back_to_back_launches_match_single_launches():
     assert not dt.status.cpu().numpy().any()
 
 
+@pytest.mark.parametrize("tck", TC_KERNELS)
 @pytest.mark.parametrize("seed", range(6))
-def test_attn_tc_random_batches_and_splits(seed):
+def test_attn_tc_random_batches_and_splits(seed, tck):
     """Random batches (ragged trees and prefixes around the tile edges), head groupings and forced
     splits through the tensor-core kernel: oracle parity, bit-identical reruns, clean status words."""
     rng = np.random.default_rng(9000 + seed)
@@ -555,11 +560,11 @@ def test_attn_tc_random_batches_and_splits(seed):
         ref = oracle_attn(tb, Hkv * G, Hkv, 128, q, k, v)
         dt = H.DevTrees(tb)
         hc = bool(rng.integers(0, 2))
-        out, rc = H.run_attn(dt, Hkv * G, Hkv, 128, q, k, v, kernel=binding.ATTN_TC, n_splits=splits, check=False,
+        out, rc = H.run_attn(dt, Hkv * G, Hkv, 128, q, k, v, kernel=tck, n_splits=splits, check=False,
                              host_copies=hc)
         tc_or_skip(rc)
         H.assert_attn_close(out, ref, tb.node_off)
-        again, _ = H.run_attn(dt, Hkv * G, Hkv, 128, q, k, v, kernel=binding.ATTN_TC, n_splits=splits, host_copies=hc)
+        again, _ = H.run_attn(dt, Hkv * G, Hkv, 128, q, k, v, kernel=tck, n_splits=splits, host_copies=hc)
         np.testing.assert_array_equal(out, again)
         assert not dt.status.cpu().numpy().any()
 
