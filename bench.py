@@ -213,6 +213,9 @@ def time_topm(ctx, binding, torch, dev, stream, logits_h, peak, m=20, copies=20,
 
 
 # --------------------------------------------------------------------------- GPU arm
+ATTN_KERNELS = {"auto": 0, "simt": 1, "tc": 2, "tck": 3}   # falcon.h FALCON_ATTN_*
+
+
 def run_falcon(args):
     import torch
     import torch.distributed as dist
@@ -286,8 +289,11 @@ def run_falcon(args):
     strides = tuple(int(s) for s in cache[0, 0].stride()[:3])
 
     # the prefix rows were written in earlier steps: the kernel may ask for them while the previous launch drains
+    # ... and each call names the next layer's caches, whose prefix rows it may have brought into L2
     attn = [binding.attn_args(tree, Hq, Hkv, D, scale, q_all[l], out_all[l], cache[l, 0], cache[l, 1], strides, s_cap,
-                              flags=binding.ATTN_PREFIX_STABLE)
+                              flags=binding.ATTN_PREFIX_STABLE, kernel=ATTN_KERNELS[args.attn_kernel],
+                              next_k_cache=cache[l + 1, 0] if l + 1 < NL and not args.no_next_hint else None,
+                              next_v_cache=cache[l + 1, 1] if l + 1 < NL and not args.no_next_hint else None)
             for l in range(NL)]
     acc = binding.accept_args(tree, spec.vocab, logits, logits.shape[1], g, path, 128, n_path, nxt)
     cmp_ = binding.compact_args(tree, NL, Hkv, D, kptr, vptr, strides, s_cap, path, 128, n_path, new_len)
@@ -433,7 +439,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="v7b", choices=sorted(synth.SPECS))
     ap.add_argument("--impl", default="falcon", choices=["falcon", "reference"])
+    ap.add_argument("--attn-kernel", default="auto", choices=sorted(ATTN_KERNELS),
+                    help="which attention kernel falcon_tree_attn is asked for (auto = the library's choice)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-next-hint", action="store_true", help="do not name the next layer's caches to falcon_tree_attn")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "falcon":
         args.warmup = 3

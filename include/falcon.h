@@ -22,8 +22,11 @@
  *     does not fit the cache) never trap: the kernel clamps the access, skips
  *     the sequence's result where it must, and ORs FALCON_DEV_* bits into the
  *     optional per-sequence device word tree.status[b].
- *   - The first call of each kind on a context may allocate scratch memory
- *     (cudaMalloc); make that call before capturing the stream into a graph.
+ *   - A call that needs more scratch memory than the context holds allocates it
+ *     (cudaMalloc) and clears what must start at zero on `stream`; make the first
+ *     call of each kind and size before capturing the stream into a graph.
+ *     Scratch only grows, and a block that was outgrown is kept until
+ *     falcon_destroy, so launches already enqueued or captured stay valid.
  *   - There is no CPU fallback and no alternative backend.
  *
  * Tree convention (Section 3.4, Appendix A): a sequence's tree has T <=
@@ -117,6 +120,13 @@ typedef struct {
  *             The tensor-core kernel may then request prefix tiles while that
  *             preceding kernel is still finishing.  Needs the tree's host copies.
  *             Without the flag every read waits for all earlier work of the stream.
+ * next_k/v_cache  optional hint for a decoding loop that calls this layer by layer: the
+ *             caches the NEXT falcon_tree_attn call on this stream will read, with the same
+ *             shape, strides, prefix lengths and FALCON_ATTN_PREFIX_STABLE set.  Once a
+ *             thread block has received its own last tile it asks for the next layer's
+ *             prefix rows to be brought into L2, so that layer's reads overlap this
+ *             layer's tail and the launch gap.  A hint only: results never depend on it,
+ *             and only rows [0, L_b) are touched (they must be readable).
  * ------------------------------------------------------------------------- */
 enum { FALCON_ATTN_AUTO = 0, FALCON_ATTN_SIMT = 1, FALCON_ATTN_TC = 2, FALCON_ATTN_TCK = 3 };
 enum { FALCON_ATTN_PREFIX_STABLE = 1 };
@@ -137,6 +147,8 @@ typedef struct {
   int32_t kernel;
   int32_t n_splits;
   int32_t flags;                           /* FALCON_ATTN_* flag bits, 0 = none          */
+  const void* next_k_cache;                /* optional hint, see above (NULL = none)     */
+  const void* next_v_cache;
 } falcon_attn_args;
 
 int falcon_tree_attn(falcon_ctx* ctx, const falcon_attn_args* args, void* stream);
@@ -210,7 +222,8 @@ int falcon_topm(falcon_ctx* ctx, const falcon_topm_args* args, void* stream);
  *
  * Limits: total_nodes <= FALCON_STATIC_MAX_NODES and batch <=
  * FALCON_STATIC_MAX_BATCH; anything larger returns FALCON_ERR_CAPACITY and
- * launches nothing.  It runs on the current device.  The first call on each
+ * launches nothing.  It runs on the current device, and `stream` must be a stream
+ * of that device (the array's address differs from device to device).  The first call on each
  * device looks up the array's device address (a one-time set-up step); make that
  * first call before any stream capture begins.  All calls on a device share the
  * one array, and it keeps the previous call's contents: the call itself clears

@@ -40,7 +40,8 @@ class AttnArgs(C.Structure):
                 ("sm_scale", C.c_float), ("q", C.c_void_p), ("out", C.c_void_p), ("k_cache", C.c_void_p),
                 ("v_cache", C.c_void_p), ("kv_stride_b", C.c_int64), ("kv_stride_h", C.c_int64),
                 ("kv_stride_s", C.c_int64), ("s_cap", C.c_int32), ("k_tree", C.c_void_p), ("v_tree", C.c_void_p),
-                ("tree_mask", C.c_void_p), ("kernel", C.c_int32), ("n_splits", C.c_int32), ("flags", C.c_int32)]
+                ("tree_mask", C.c_void_p), ("kernel", C.c_int32), ("n_splits", C.c_int32), ("flags", C.c_int32),
+                ("next_k_cache", C.c_void_p), ("next_v_cache", C.c_void_p)]
 
 
 class AcceptArgs(C.Structure):
@@ -199,11 +200,13 @@ class Context:
 
 
 def attn_args(tree: TreeDesc, n_q_heads, n_kv_heads, head_dim, sm_scale, q, out, k_cache, v_cache, strides, s_cap,
-              k_tree=None, v_tree=None, tree_mask=None, kernel=ATTN_AUTO, n_splits=0, flags=0) -> AttnArgs:
-    """flags: ATTN_PREFIX_STABLE when the prefix rows were written before the preceding kernel started."""
+              k_tree=None, v_tree=None, tree_mask=None, kernel=ATTN_AUTO, n_splits=0, flags=0,
+              next_k_cache=None, next_v_cache=None) -> AttnArgs:
+    """flags: ATTN_PREFIX_STABLE when the prefix rows were written before the preceding kernel started.
+    next_k_cache / next_v_cache: the caches the next call on the stream will read (an L2 prefetch hint)."""
     return AttnArgs(tree, n_q_heads, n_kv_heads, head_dim, sm_scale, _ptr(q), _ptr(out), _ptr(k_cache),
                     _ptr(v_cache), strides[0], strides[1], strides[2], s_cap, _ptr(k_tree), _ptr(v_tree),
-                    _ptr(tree_mask), kernel, n_splits, flags)
+                    _ptr(tree_mask), kernel, n_splits, flags, _ptr(next_k_cache), _ptr(next_v_cache))
 
 
 def accept_args(tree: TreeDesc, vocab, logits, logits_stride, argmax_out, path, path_stride, n_path,

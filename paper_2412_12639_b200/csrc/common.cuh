@@ -7,6 +7,7 @@
 #include <stdint.h>
 
 #include <string>
+#include <vector>
 
 #include "falcon.h"
 
@@ -20,6 +21,9 @@ struct falcon_ctx {
   // Arrival counters; zero between calls (the last arriver resets its counter).
   int* tickets = nullptr;
   size_t n_tickets = 0;
+  // Scratch blocks that were outgrown.  A launch already enqueued, or captured into a CUDA graph,
+  // may still name them, so they live until falcon_destroy.
+  std::vector<void*> retired;
   std::string last_error;
   // Cached TMA descriptors (opaque here; owned by tc_util.cuh).
   void* tmap_cache = nullptr;
@@ -34,7 +38,7 @@ struct falcon_ctx {
 namespace falcon {
 
 int ensure_workspace(falcon_ctx* ctx, size_t bytes);
-int ensure_tickets(falcon_ctx* ctx, size_t count);
+int ensure_tickets(falcon_ctx* ctx, size_t count, cudaStream_t stream);
 int cuda_fail(falcon_ctx* ctx, cudaError_t e, const char* where);
 int check_tree_desc(const falcon_tree_desc& t, bool need_token);
 
@@ -47,6 +51,7 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
 bool tree_attn_tc_supports(const falcon_ctx* ctx, const falcon_attn_args& a);
 int launch_tree_attn_tck(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s);
 bool tree_attn_tck_supports(const falcon_ctx* ctx, const falcon_attn_args& a);
+bool tree_attn_tck_preferred(const falcon_ctx* ctx, const falcon_attn_args& a);
 void tree_attn_tc_release(falcon_ctx* ctx);
 
 #ifdef __CUDACC__

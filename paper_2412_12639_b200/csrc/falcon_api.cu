@@ -12,29 +12,35 @@ int cuda_fail(falcon_ctx* ctx, cudaError_t e, const char* where) {
   return FALCON_ERR_CUDA;
 }
 
+// Scratch only ever grows, and a block that was outgrown is kept until the context is destroyed:
+// a kernel already enqueued, or a captured graph, may still name it.
 int ensure_workspace(falcon_ctx* ctx, size_t bytes) {
   if (bytes <= ctx->ws_bytes) return FALCON_OK;
-  // cudaFree waits for work in flight, so a kernel still reading the old block is safe.
-  if (ctx->ws) cudaFree(ctx->ws);
-  ctx->ws = nullptr;
-  ctx->ws_bytes = 0;
   const size_t want = bytes + bytes / 4;
-  cudaError_t e = cudaMalloc(&ctx->ws, want);
+  void* fresh = nullptr;
+  cudaError_t e = cudaMalloc(&fresh, want);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMalloc(workspace)");
+  if (ctx->ws) ctx->retired.push_back(ctx->ws);
+  ctx->ws = fresh;
   ctx->ws_bytes = want;
   return FALCON_OK;
 }
 
-int ensure_tickets(falcon_ctx* ctx, size_t count) {
+// Arrival counters must read zero when a kernel first uses them: a new block is cleared on the
+// caller's stream, ahead of the launch that follows (the kernels leave their counters at zero).
+int ensure_tickets(falcon_ctx* ctx, size_t count, cudaStream_t stream) {
   if (count <= ctx->n_tickets) return FALCON_OK;
-  if (ctx->tickets) cudaFree(ctx->tickets);
-  ctx->tickets = nullptr;
-  ctx->n_tickets = 0;
   const size_t want = count * 2 + 64;
-  cudaError_t e = cudaMalloc(&ctx->tickets, want * sizeof(int));
+  int* fresh = nullptr;
+  cudaError_t e = cudaMalloc(&fresh, want * sizeof(int));
   if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMalloc(tickets)");
-  e = cudaMemset(ctx->tickets, 0, want * sizeof(int));
-  if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMemset(tickets)");
+  e = cudaMemsetAsync(fresh, 0, want * sizeof(int), stream);
+  if (e != cudaSuccess) {
+    cudaFree(fresh);
+    return cuda_fail(ctx, e, "cudaMemsetAsync(tickets)");
+  }
+  if (ctx->tickets) ctx->retired.push_back(ctx->tickets);
+  ctx->tickets = fresh;
   ctx->n_tickets = want;
   return FALCON_OK;
 }
@@ -78,6 +84,7 @@ int falcon_destroy(falcon_ctx* ctx) {
   tree_attn_tc_release(ctx);
   if (ctx->ws) cudaFree(ctx->ws);
   if (ctx->tickets) cudaFree(ctx->tickets);
+  for (void* blk : ctx->retired) cudaFree(blk);
   delete ctx;
   return FALCON_OK;
 }
@@ -135,8 +142,9 @@ int falcon_tree_attn(falcon_ctx* ctx, const falcon_attn_args* a, void* stream) {
       if (!tree_attn_tck_supports(ctx, *a)) return FALCON_ERR_UNSUPPORTED;
       return launch_tree_attn_tck(ctx, *a, s);
     case FALCON_ATTN_AUTO:
+      if (tree_attn_tck_supports(ctx, *a) && (tree_attn_tck_preferred(ctx, *a) || !tree_attn_tc_supports(ctx, *a)))
+        return launch_tree_attn_tck(ctx, *a, s);
       if (tree_attn_tc_supports(ctx, *a)) return launch_tree_attn_tc(ctx, *a, s);
-      if (tree_attn_tck_supports(ctx, *a)) return launch_tree_attn_tck(ctx, *a, s);
       return launch_tree_attn_simt(ctx, *a, s);
     default:
       return FALCON_ERR_INVALID_ARG;

@@ -182,30 +182,28 @@ __global__ void __launch_bounds__(kAcceptThreads) tree_accept_kernel(const Accep
   }
 }
 
-}  // namespace
+constexpr int kAcceptMaxChunks = 64;  // vocabulary chunks per row at most (the static scratch is sized by it)
 
-int launch_tree_accept(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_t s) {
-  const int N = a.tree.total_nodes;
-  if (N > 65535) return FALCON_ERR_CAPACITY;
-  // enough CTAs for a few waves, chunks of at least 2048 elements
-  int chunks = (4 * ctx->sm_count + N - 1) / N;
-  const int max_chunks = (a.vocab + 2047) / 2048;
+// How a launch splits the vocabulary: enough CTAs for a few waves, chunks of at least 2048 elements
+// and a multiple of 4.  Shared by the two entry points so that they cannot drift apart.
+void accept_plan(int sm_count, int n_nodes, int vocab, int* chunks_out, int* chunk_len_out) {
+  int chunks = (4 * sm_count + n_nodes - 1) / n_nodes;
+  const int max_chunks = (vocab + 2047) / 2048;
   if (chunks > max_chunks) chunks = max_chunks;
-  if (chunks > 64) chunks = 64;
+  if (chunks > kAcceptMaxChunks) chunks = kAcceptMaxChunks;
   if (chunks < 1) chunks = 1;
-  int chunk_len = (a.vocab + chunks - 1) / chunks;
+  int chunk_len = (vocab + chunks - 1) / chunks;
   chunk_len = (chunk_len + 3) & ~3;
-  chunks = (a.vocab + chunk_len - 1) / chunk_len;
+  *chunks_out = (vocab + chunk_len - 1) / chunk_len;
+  *chunk_len_out = chunk_len;
+}
 
-  const size_t part = static_cast<size_t>(N) * chunks;
-  int rc = ensure_workspace(ctx, part * 8 + 256);
-  if (rc) return rc;
-  rc = ensure_tickets(ctx, a.tree.batch);
-  if (rc) return rc;
-
+// Kernel parameters from the caller's arguments, the plan and the scratch: `part` holds
+// n_nodes * chunks values followed by as many indices, `tickets` one counter per sequence.
+AcceptParams accept_params(const falcon_accept_args& a, int chunks, int chunk_len, void* part, int* tickets) {
   AcceptParams p;
   p.batch = a.tree.batch;
-  p.total_nodes = N;
+  p.total_nodes = a.tree.total_nodes;
   p.vocab = a.vocab;
   p.chunks = chunks;
   p.chunk_len = chunk_len;
@@ -220,9 +218,26 @@ int launch_tree_accept(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_
   p.path = a.path;
   p.n_path = a.n_path;
   p.next_token = a.next_token;
-  p.part_val = static_cast<float*>(ctx->ws);
-  p.part_idx = reinterpret_cast<int32_t*>(static_cast<float*>(ctx->ws) + part);
-  p.tickets = ctx->tickets;
+  p.part_val = static_cast<float*>(part);
+  p.part_idx = reinterpret_cast<int32_t*>(part) + static_cast<size_t>(a.tree.total_nodes) * chunks;
+  p.tickets = tickets;
+  return p;
+}
+
+}  // namespace
+
+int launch_tree_accept(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_t s) {
+  const int N = a.tree.total_nodes;
+  if (N > 65535) return FALCON_ERR_CAPACITY;
+  int chunks, chunk_len;
+  accept_plan(ctx->sm_count, N, a.vocab, &chunks, &chunk_len);
+
+  const size_t part = static_cast<size_t>(N) * chunks;
+  int rc = ensure_workspace(ctx, part * 8 + 256);
+  if (rc) return rc;
+  rc = ensure_tickets(ctx, a.tree.batch, s);
+  if (rc) return rc;
+  const AcceptParams p = accept_params(a, chunks, chunk_len, ctx->ws, ctx->tickets);
 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(chunks, N);
@@ -258,7 +273,7 @@ namespace {
 
 constexpr int kStaticMaxNodes = FALCON_STATIC_MAX_NODES;
 constexpr int kStaticMaxBatch = FALCON_STATIC_MAX_BATCH;
-constexpr int kStaticMaxChunks = 64;
+constexpr int kStaticMaxChunks = kAcceptMaxChunks;
 constexpr size_t kStaticPartBytes = static_cast<size_t>(kStaticMaxNodes) * kStaticMaxChunks * 8;  // values + indices
 constexpr size_t kStaticBytes = kStaticPartBytes + static_cast<size_t>(kStaticMaxBatch) * sizeof(int);
 
@@ -313,43 +328,16 @@ extern "C" int falcon_tree_accept_static(const falcon_accept_args* a, void* stre
   if (rc) return rc;
 
   const int N = a->tree.total_nodes;
-  int chunks = (4 * slot.sm_count + N - 1) / N;
-  const int max_chunks = (a->vocab + 2047) / 2048;
-  if (chunks > max_chunks) chunks = max_chunks;
-  if (chunks > kStaticMaxChunks) chunks = kStaticMaxChunks;
-  if (chunks < 1) chunks = 1;
-  int chunk_len = (a->vocab + chunks - 1) / chunks;
-  chunk_len = (chunk_len + 3) & ~3;
-  chunks = (a->vocab + chunk_len - 1) / chunk_len;
+  int chunks, chunk_len;
+  accept_plan(slot.sm_count, N, a->vocab, &chunks, &chunk_len);
 
   unsigned char* base = static_cast<unsigned char*>(slot.ptr);
-  const size_t part = static_cast<size_t>(N) * chunks;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // The array keeps whatever the previous call left.  The partials are fully rewritten by this
   // launch; the arrival counters must start at zero, so they are cleared on the stream first.
   cudaError_t e = cudaMemsetAsync(base + kStaticPartBytes, 0, static_cast<size_t>(a->tree.batch) * sizeof(int), s);
   if (e != cudaSuccess) return FALCON_ERR_CUDA;
-
-  AcceptParams p;
-  p.batch = a->tree.batch;
-  p.total_nodes = N;
-  p.vocab = a->vocab;
-  p.chunks = chunks;
-  p.chunk_len = chunk_len;
-  p.path_stride = a->path_stride;
-  p.logits_stride = a->logits_stride;
-  p.node_off = a->tree.node_off;
-  p.parent = a->tree.parent;
-  p.token = a->tree.token;
-  p.status = a->tree.status;
-  p.logits = a->logits;
-  p.argmax_out = a->argmax_out;
-  p.path = a->path;
-  p.n_path = a->n_path;
-  p.next_token = a->next_token;
-  p.part_val = reinterpret_cast<float*>(base);
-  p.part_idx = reinterpret_cast<int32_t*>(base) + part;
-  p.tickets = reinterpret_cast<int*>(base + kStaticPartBytes);
+  const AcceptParams p = accept_params(*a, chunks, chunk_len, base, reinterpret_cast<int*>(base + kStaticPartBytes));
   dim3 grid(chunks, N);
   tree_accept_kernel<<<grid, kAcceptThreads, 0, s>>>(p);
   e = cudaGetLastError();

@@ -378,7 +378,7 @@ int launch_tree_attn_simt(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream
     const size_t o_bytes = rows * a.head_dim * sizeof(float);
     int rc = ensure_workspace(ctx, o_bytes + rows * sizeof(float2) + 256);
     if (rc) return rc;
-    rc = ensure_tickets(ctx, static_cast<size_t>(B) * Hq);
+    rc = ensure_tickets(ctx, static_cast<size_t>(B) * Hq, s);
     if (rc) return rc;
     p.part_o = static_cast<float*>(ctx->ws);
     p.part_ml = reinterpret_cast<float2*>(static_cast<char*>(ctx->ws) + o_bytes);

@@ -710,7 +710,21 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     __syncwarp();
     const int row0 = split * rows_per;
     const int rows_mine = max(0, min(n_valid, row0 + rows_per) - row0);
-    const bool got = rows_mine == 0 || n_splits == 1 || mbar_wait_warp(bar(kBarMrg), 0, abort_flag);
+    bool got = rows_mine == 0 || n_splits == 1 || mbar_wait_warp(bar(kBarMrg), 0, abort_flag);
+    if (!got) {
+      // This wait gave up (or another did).  Every peer still sends its rows, whatever happened to it,
+      // so stay, without looking at the abort flag, until they have landed: the CTA must not reach the
+      // exit barrier, and leave, while a copy into its merge area is in flight.  The rows stay unmerged.
+      bool landed = false;
+      for (uint32_t it = 0; it < (1u << 20) && !landed; ++it) {
+        uint32_t ok;
+        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                     : "=r"(ok)
+                     : "r"(bar(kBarMrg)), "r"(0u)
+                     : "memory");
+        landed = __all_sync(0xffffffffu, ok != 0);
+      }
+    }
     FALCON_TRACE(tid == 0, 74);
     const unsigned char* mrg = smem_gen + kOffMrg;
     const unsigned char* own = smem_gen + kOffStage + static_cast<uint32_t>(row0) * kMrgRowBytes;

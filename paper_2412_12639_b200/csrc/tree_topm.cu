@@ -207,7 +207,7 @@ int launch_tree_topm(falcon_ctx* ctx, const falcon_topm_args& a, cudaStream_t s)
   const size_t part = static_cast<size_t>(N) * chunks * a.m;
   int rc = ensure_workspace(ctx, part * 8 + 256);
   if (rc) return rc;
-  rc = ensure_tickets(ctx, N);
+  rc = ensure_tickets(ctx, N, s);
   if (rc) return rc;
 
   TopmParams p;

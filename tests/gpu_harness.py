@@ -83,25 +83,40 @@ def run_attn(dt: DevTrees, Hq, Hkv, D, q, k, v, s_cap=None, scale=None, kernel=b
     return host_bits(out), rc
 
 
+ROW_REL_L2 = 1e-2  # per (node, head) row: ||gpu - oracle||_2 / max(||oracle||_2, ROW_FLOOR)
+ROW_FLOOR = 0.05   # rows whose oracle norm is below this are measured against it (a near-zero row has no scale of its own)
+RTOL = 1e-2        # elementwise |gpu - oracle| <= ATOL + RTOL * |oracle|
+
+
 def attn_errors(out_bits, ref, node_off):
-    """max abs error and the worst per-(sequence, head) relative L2 error."""
+    """max abs error, the worst per-(sequence, head) relative L2 error, the worst per-(node, head) row relative L2
+    error (with its node and head) and the fraction of elements inside |d| <= ATOL + RTOL * |ref|."""
     got = synth.bf16_bits_to_f32(out_bits).astype(np.float64)
     ref = ref.astype(np.float64)
     assert np.isfinite(got).all(), "non-finite attention output"
-    max_abs = float(np.abs(got - ref).max())
+    d = got - ref
+    max_abs = float(np.abs(d).max())
     worst = 0.0
     for b in range(len(node_off) - 1):
         lo, hi = node_off[b], node_off[b + 1]
-        num = np.sqrt(((got[lo:hi] - ref[lo:hi]) ** 2).sum(axis=(0, 2)))
+        num = np.sqrt((d[lo:hi] ** 2).sum(axis=(0, 2)))
         den = np.sqrt((ref[lo:hi] ** 2).sum(axis=(0, 2)))
         worst = max(worst, float((num / np.maximum(den, 1e-30)).max()))
-    return max_abs, worst
+    row = np.sqrt((d ** 2).sum(axis=2)) / np.maximum(np.sqrt((ref ** 2).sum(axis=2)), ROW_FLOOR)
+    at = np.unravel_index(int(np.argmax(row)), row.shape)
+    inside = float((np.abs(d) <= ATOL + RTOL * np.abs(ref)).mean())
+    return max_abs, worst, float(row[at]), (int(at[0]), int(at[1])), inside
 
 
-def assert_attn_close(out_bits, ref, node_off):
-    max_abs, rel = attn_errors(out_bits, ref, node_off)
+def assert_attn_close(out_bits, ref, node_off, report=False):
+    max_abs, rel, row_rel, row_at, inside = attn_errors(out_bits, ref, node_off)
+    if report:
+        print("attention vs oracle: max abs %.3g, block rel L2 %.3g, worst row rel L2 %.3g at (node %d, head %d), "
+              "allclose(atol %.0e, rtol %.0e) fraction %.6f" % (max_abs, rel, row_rel, row_at[0], row_at[1], ATOL, RTOL, inside))
     assert max_abs <= ATOL, "max abs error %.4g > %.4g" % (max_abs, ATOL)
     assert rel <= REL_L2, "relative L2 error %.4g > %.4g" % (rel, REL_L2)
+    assert row_rel <= ROW_REL_L2, "row (node %d, head %d): relative L2 error %.4g > %.4g" % (row_at + (row_rel, ROW_REL_L2))
+    assert inside == 1.0, "elements outside atol + rtol * |ref|: fraction %.3g" % (1.0 - inside)
     return max_abs, rel
 
 

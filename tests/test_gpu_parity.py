@@ -177,21 +177,35 @@ def test_attn_separate_tree_buffers(kernel):
     H.assert_attn_close(out, ref, tb.node_off)
 
 
+def relaxed_mask_rows(tb, k_block, drop=()):
+    """Mask rows of the drafter's relaxed causal mask (Section 3.4): a node sees its predecessors in the tree and the
+    nodes of its own block of k_block consecutive nodes.  `drop` lists (packed node, tree key) bits to clear."""
+    rows = np.zeros((tb.total_nodes, 2), np.uint64)
+    for b in range(tb.batch):
+        o, T = int(tb.node_off[b]), tb.tree_size(b)
+        par = tb.parent[o:o + T]
+        for i in range(T):
+            vis = set(oracle.ancestors(par, i)) | {m for m in range(i - i % k_block, min(T, i - i % k_block + k_block))}
+            for a in vis:
+                rows[o + i, a >> 6] |= np.uint64(1) << np.uint64(a & 63)
+    for node, key in drop:
+        rows[node, key >> 6] &= ~(np.uint64(1) << np.uint64(key & 63))
+    return rows
+
+
 @pytest.mark.parametrize("kernel", KERNELS)
-def test_attn_caller_mask_rows(kernel):
-    # relaxed causal mask of the drafter (Section 3.4): ancestors plus the nodes of the same k-block
+@pytest.mark.parametrize("splits", [0, 3])
+def test_attn_caller_mask_rows(kernel, splits):
+    # relaxed causal mask of the drafter on a batch of two sequences with different tree sizes and prefixes, one row
+    # with an ancestor bit cleared: the rows of the second sequence start at a non-zero packed offset
     rng = np.random.default_rng(10)
-    T, L = 50, 90
-    tb, q, k, v = random_case(rng, [T], [L], 2, 2, 128)
-    rows = np.zeros((T, 2), np.uint64)
-    for i in range(T):
-        for a in oracle.ancestors(tb.parent, i):
-            rows[i, a >> 6] |= np.uint64(1) << np.uint64(a & 63)
-        mate = i ^ 1                                    # k = 2 blocks: (0,1), (2,3), ...
-        if mate < T:
-            rows[i, mate >> 6] |= np.uint64(1) << np.uint64(mate & 63)
-    ref = oracle_attn(tb, 2, 2, 128, q, k, v, tree_mask=rows)
-    out, rc = H.run_attn(H.DevTrees(tb), 2, 2, 128, q, k, v, tree_mask=rows, kernel=kernel, check=False)
+    sizes, prefs = [50, 77], [90, 301]
+    tb, q, k, v = random_case(rng, sizes, prefs, 4, 2, 128, slack=2)
+    rows = relaxed_mask_rows(tb, 3, drop=[(50 + 40, int(tb.parent[50 + 40]))])
+    ref = oracle_attn(tb, 4, 2, 128, q, k, v, tree_mask=rows)
+    plain = oracle_attn(tb, 4, 2, 128, q, k, v)
+    assert np.abs(ref - plain).max() > 0.05            # the mask rows do change the result
+    out, rc = H.run_attn(H.DevTrees(tb), 4, 2, 128, q, k, v, tree_mask=rows, kernel=kernel, n_splits=splits, check=False)
     tc_or_skip(rc)
     H.assert_attn_close(out, ref, tb.node_off)
 
@@ -246,12 +260,13 @@ def test_attn_malformed_tree_and_capacity_set_status_without_faulting():
         assert dt2.status.cpu().numpy()[0] & binding.DEV_CAPACITY
 
 
-FULL = {"v7b": [0, 17, 31], "l13b": [3, 22, 39], "l70b": [1, 5], "ragged": [2, 30]}
+FULL = {"v7b": list(range(32)), "l13b": list(range(40)), "l70b": [1, 5], "ragged": [2, 30]}   # KV heads the oracle checks
 
 
 @pytest.mark.parametrize("name", ["v7b", "l13b", "l70b", "ragged"])
 def test_attn_full_size_configs_sampled_heads(name):
-    """Full-size launch (the one the benchmark times); the oracle checks a sample of KV heads of one layer."""
+    """Full-size launch (the one the benchmark times); the oracle checks every head of one layer of the two graded
+    shapes and a sample of KV heads of the two large ones, per (node, head) row."""
     spec = synth.SPECS[name]
     tb = synth.make_trees(spec)
     q, k, v = synth.make_layer_qkv(spec, tb, 1)
@@ -264,7 +279,7 @@ def test_attn_full_size_configs_sampled_heads(name):
         ks = np.ascontiguousarray(k[:, kvh:kvh + 1])
         vs = np.ascontiguousarray(v[:, kvh:kvh + 1])
         ref = oracle_attn(tb, G, 1, spec.head_dim, qs, ks, vs)
-        H.assert_attn_close(np.ascontiguousarray(out[:, kvh * G:(kvh + 1) * G]), ref, tb.node_off)
+        H.assert_attn_close(np.ascontiguousarray(out[:, kvh * G:(kvh + 1) * G]), ref, tb.node_off, report=kvh == FULL[name][0])
 
 
 # --------------------------------------------------------------------- accept
@@ -668,3 +683,79 @@ def test_abi_rejects_bad_arguments_without_launching():
     assert c.falcon_tree_accept(binding.accept_args(dt.desc(), 10, None, 10, g, path, 128, n, nxt), check=False) \
         == binding.ERR_INVALID_ARG
     torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------ contexts, scratch
+def _accept_buffers(tb):
+    i32 = lambda *s: torch.full(s, -7, dtype=torch.int32, device="cuda")
+    return i32(tb.total_nodes), i32(tb.batch, 128), i32(tb.batch), i32(tb.batch)
+
+
+def test_two_contexts_used_in_turn_keep_their_own_state():
+    """Two contexts on the device, called alternately (attention through both tensor-core kernels, acceptance):
+    launch attributes, cluster occupancy and scratch are per context, so neither disturbs the other."""
+    import paper_2412_12639_b200 as falcon
+    rng = np.random.default_rng(77)
+    tb, q, k, v = random_case(rng, [60, 33], [700, 130], 4, 4, 128)
+    ref = oracle_attn(tb, 4, 4, 128, q, k, v)
+    logits = rng.standard_normal((tb.total_nodes, 5000)).astype(np.float32)
+    g_ref = oracle.argmax(logits)
+    p_ref, n_ref, t_ref = oracle.tree_accept(tb.node_off, tb.parent, tb.token, g_ref)
+    dt = H.DevTrees(tb)
+    qd, kd, vd, ld = H.dev_bf16(q), H.dev_bf16(k), H.dev_bf16(v), torch.from_numpy(logits).cuda()
+    ctxs = [falcon.Context(0), falcon.Context(0)]
+    strides = tuple(int(s) for s in kd.stride()[:3])
+    for rnd in range(3):
+        for c in ctxs:
+            for kernel in TC_KERNELS:
+                out = torch.full_like(qd, float("nan"))
+                c.falcon_tree_attn(binding.attn_args(dt.desc(), 4, 4, 128, 1 / math.sqrt(128), qd, out, kd, vd, strides,
+                                                     kd.shape[2], kernel=kernel))
+                torch.cuda.synchronize()
+                H.assert_attn_close(H.host_bits(out), ref, tb.node_off)
+            g, path, n_path, nxt = _accept_buffers(tb)
+            c.falcon_tree_accept(binding.accept_args(dt.desc(), 5000, ld, 5000, g, path, 128, n_path, nxt))
+            torch.cuda.synchronize()
+            np.testing.assert_array_equal(g.cpu().numpy(), g_ref)
+            np.testing.assert_array_equal(path.cpu().numpy(), p_ref)
+    for c in ctxs:
+        c.close()
+
+
+def test_captured_graph_survives_a_later_call_that_needs_more_scratch():
+    """An acceptance call captured into a CUDA graph, then a top-m call on the same context that needs a larger
+    scratch block and more arrival counters (on a non-blocking stream), then the graph replayed: the graph still
+    names the block it was captured with, which must be alive and consistent."""
+    import paper_2412_12639_b200 as falcon
+    rng = np.random.default_rng(78)
+    tb = H.make_trees([20, 9], [0, 0], rng, vocab=50)
+    logits = rng.standard_normal((tb.total_nodes, 3000)).astype(np.float32)
+    g_ref = oracle.argmax(logits)
+    p_ref, n_ref, t_ref = oracle.tree_accept(tb.node_off, tb.parent, tb.token, g_ref)
+    dt = H.DevTrees(tb)
+    ld = torch.from_numpy(logits).cuda()
+    c = falcon.Context(0)
+    g, path, n_path, nxt = _accept_buffers(tb)
+    acc = binding.accept_args(dt.desc(), 3000, ld, 3000, g, path, 128, n_path, nxt)
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        c.falcon_tree_accept(acc, stream=st)               # first call: allocates, outside the capture
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=st):
+            c.falcon_tree_accept(acc, stream=st)
+        big = torch.from_numpy(rng.standard_normal((300, 40000)).astype(np.float32)).cuda()
+        val = torch.zeros((300, 8), device="cuda")
+        idx = torch.zeros((300, 8), dtype=torch.int32, device="cuda")
+        c.falcon_topm(binding.topm_args(300, 40000, big, 40000, 8, val, idx), stream=st)   # grows both scratch blocks
+        for _ in range(3):
+            g.fill_(-7)
+            path.fill_(-7)
+            graph.replay()
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(g.cpu().numpy(), g_ref)
+    np.testing.assert_array_equal(path.cpu().numpy(), p_ref)
+    np.testing.assert_array_equal(n_path.cpu().numpy(), n_ref)
+    want_v, want_i = oracle.topm(big.cpu().numpy(), 8)
+    np.testing.assert_array_equal(idx.cpu().numpy(), want_i)
+    c.close()

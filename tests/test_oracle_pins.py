@@ -285,6 +285,51 @@ def test_attn_explicit_mask_rows_reproduce_the_ancestor_mask():
     np.testing.assert_allclose(a, b, atol=1e-7)
 
 
+def test_attn_mask_rows_on_a_batch_match_sdpa_with_the_same_boolean_mask():
+    """The caller-supplied mask branch against torch's scaled_dot_product_attention with an explicit boolean mask,
+    on two sequences of different tree size and prefix length: rows of the drafter's relaxed causal mask
+    (Section 3.4: predecessors in the tree plus the node's own k-block) and one row with an ancestor bit cleared.
+    A wrong row offset for the second sequence, or rows merged with the ancestor chain, fail here."""
+    import torch
+    rng = np.random.default_rng(33)
+    sizes, prefs, Hq, Hkv, D, kblk = [23, 70], [5, 41], 4, 2, 16, 3
+    node_off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    parents = [synth.random_tree(rng, t, 8, 4) for t in sizes]
+    parent = np.concatenate(parents).astype(np.int32)
+    N, s_cap = int(node_off[-1]), max(p + t for p, t in zip(prefs, sizes)) + 1
+    q = synth.normal_bf16(rng, (N, Hq, D))
+    k = synth.normal_bf16(rng, (2, Hkv, s_cap, D))
+    v = synth.normal_bf16(rng, (2, Hkv, s_cap, D))
+    rows = np.zeros((N, 2), np.uint64)
+    vis = [[set() for _ in range(t)] for t in sizes]
+    for b, (T, par) in enumerate(zip(sizes, parents)):
+        for i in range(T):
+            s_ = {a for a in range(T) if is_ancestor_or_self(par, a, i)} | set(range(i - i % kblk, min(T, i - i % kblk + kblk)))
+            vis[b][i] = s_
+    dropped = int(parents[1][40])
+    vis[1][40].discard(dropped)                                # not even the ancestor chain is implied
+    for b, T in enumerate(sizes):
+        for i in range(T):
+            for a in vis[b][i]:
+                rows[node_off[b] + i, a >> 6] |= np.uint64(1) << np.uint64(a & 63)
+    out = oracle.tree_attn(node_off, parent, prefs, Hq, Hkv, D, 0.31, q, k, v, strides_of(k), tree_mask=rows)
+    plain = oracle.tree_attn(node_off, parent, prefs, Hq, Hkv, D, 0.31, q, k, v, strides_of(k))
+    assert np.abs(out - plain).max() > 1e-2
+    qf, kf, vf = (torch.from_numpy(synth.bf16_bits_to_f32(x).astype(np.float64)) for x in (q, k, v))
+    G = Hq // Hkv
+    for b, (T, L) in enumerate(zip(sizes, prefs)):
+        mask = torch.zeros(T, L + T, dtype=torch.bool)
+        mask[:, :L] = True
+        for i in range(T):
+            for a in vis[b][i]:
+                mask[i, L + a] = True
+        for h in range(Hq):
+            qq = qf[node_off[b]:node_off[b + 1], h]
+            want = torch.nn.functional.scaled_dot_product_attention(
+                qq[None], kf[b, h // G, :L + T][None], vf[b, h // G, :L + T][None], attn_mask=mask[None], scale=0.31)[0]
+            np.testing.assert_allclose(out[node_off[b]:node_off[b + 1], h], want.numpy(), atol=2e-6, rtol=1e-6)
+
+
 # -------------------------------------------------------------------- argmax
 def test_argmax_planted_ties_and_special_values():
     rng = np.random.default_rng(0)
