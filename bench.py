@@ -48,14 +48,14 @@ def accept_bytes(spec, tb) -> int:
     return 4 * tb.total_nodes * spec.vocab + 12 * tb.total_nodes
 
 
-def recorded_traffic(workload: str):
-    """DRAM bytes per attention launch from the committed ncu summary of this workload, or None when
-    there is none or the kernel source has changed since the counters were taken."""
+def recorded_traffic(workload: str, kernel: str):
+    """DRAM bytes per attention launch from the committed ncu summary of this workload and kernel ("tc", "tck"),
+    or None when there is none or the kernel source has changed since the counters were taken."""
     import hashlib
     import re
     try:
-        text = open(os.path.join(ROOT, "profiles", "tree_attn_tc_%s_ncu.md" % workload)).read()
-        src = open(os.path.join(ROOT, "paper_2412_12639_b200", "csrc", "tree_attn_tc.cu"), "rb").read()
+        text = open(os.path.join(ROOT, "profiles", "tree_attn_%s_%s_ncu.md" % (kernel, workload))).read()
+        src = open(os.path.join(ROOT, "paper_2412_12639_b200", "csrc", "tree_attn_%s.cu" % kernel), "rb").read()
     except OSError:
         return None
     sha = re.search(r"kernel_source_sha256:\s*([0-9a-f]{64})", text)
@@ -116,20 +116,21 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- oracle timing (CPU)
-def time_oracle_step(spec, tb, logits, sample_layers: int):
-    """Runs the CPU oracle on `sample_layers` layers of attention and compaction plus the full acceptance,
-    and extrapolates one whole step.  Returns (seconds per step, threads, description)."""
+def time_oracle_step(spec, tb, logits, sample_layers: int, n_threads: int = 0):
+    """Runs the CPU oracle on `sample_layers` layers of attention and compaction plus the full acceptance.
+    With all layers this is one whole step; with fewer the per-layer time is extrapolated to the step.
+    Returns (seconds per step, threads, description, extrapolated)."""
     import oracle
     scale = 1.0 / math.sqrt(spec.head_dim)
     t_attn = t_comp = 0.0
-    g = oracle.argmax(logits)
+    g = oracle.argmax(logits, n_threads=n_threads)
     path, n_path, _ = oracle.tree_accept(tb.node_off, tb.parent, tb.token, g)
     for layer in range(sample_layers):
         q, k, v = synth.make_layer_qkv(spec, tb, layer)
         st = tuple(s // 2 for s in k.strides[:3])
         t0 = time.perf_counter()
         oracle.tree_attn(tb.node_off, tb.parent, tb.prefix_len, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, scale,
-                         q, k, v, st)
+                         q, k, v, st, n_threads=n_threads)
         t1 = time.perf_counter()
         oracle.kv_compact(tb.node_off, tb.prefix_len, spec.n_kv_heads, spec.head_dim, k, st, k.shape[2], path, n_path)
         oracle.kv_compact(tb.node_off, tb.prefix_len, spec.n_kv_heads, spec.head_dim, v, st, v.shape[2], path, n_path)
@@ -137,42 +138,72 @@ def time_oracle_step(spec, tb, logits, sample_layers: int):
         t_attn += t1 - t0
         t_comp += t2 - t1
     t0 = time.perf_counter()
-    g = oracle.argmax(logits)
+    g = oracle.argmax(logits, n_threads=n_threads)
     oracle.tree_accept(tb.node_off, tb.parent, tb.token, g)
     t_acc = time.perf_counter() - t0
     step = (t_attn + t_comp) / sample_layers * spec.n_layers + t_acc
-    desc = "%d of %d layers of attention+compaction and the full acceptance, extrapolated to one step" % (
-        sample_layers, spec.n_layers)
-    return step, oracle.max_threads(), desc
+    extrapolated = sample_layers < spec.n_layers
+    if extrapolated:
+        desc = "%d of %d layers of attention+compaction and the full acceptance, extrapolated to one step" % (
+            sample_layers, spec.n_layers)
+    else:
+        desc = "one whole step: all %d layers of attention+compaction and the acceptance" % spec.n_layers
+    threads = n_threads if n_threads > 0 else oracle.max_threads()
+    return step, threads, desc, extrapolated
 
 
-def oracle_sample_layers(spec, tb) -> int:
-    # scalar double flops of one layer of attention; aim at roughly 10-20 s on a few cores
-    flops = 4.0 * spec.head_dim * spec.n_q_heads * sum(
+def oracle_layer_flops(spec, tb) -> float:
+    """Scalar double-precision flops of one layer of oracle attention."""
+    return 4.0 * spec.head_dim * spec.n_q_heads * sum(
         tb.tree_size(b) * (int(tb.prefix_len[b]) + tb.tree_size(b)) for b in range(tb.batch))
-    return max(1, min(spec.n_layers, int(12e9 / max(flops, 1.0))))
+
+
+def oracle_sample_layers(spec, tb, budget_flops: float = 40e9) -> int:
+    """Layers of the oracle that fit a budget (about 40 GFLOP: roughly 10-30 s on a few cores); a whole step
+    when it fits (the 7B-shaped step is 34 GFLOP)."""
+    return max(1, min(spec.n_layers, int(budget_flops / max(oracle_layer_flops(spec, tb), 1.0))))
+
+
+def config_of(args, spec, tb, world: int) -> dict:
+    """The workload description both arms print, key for key."""
+    step_bytes = spec.n_layers * attn_bytes_per_layer(spec, tb) + accept_bytes(spec, tb)
+    return {"workload": args.workload, "batch": tb.batch, "n_layers": spec.n_layers, "n_q_heads": spec.n_q_heads,
+            "n_kv_heads": spec.n_kv_heads, "head_dim": spec.head_dim, "prefix_len": tb.prefix_len.tolist(),
+            "tree_nodes": np.diff(tb.node_off).tolist(), "vocab": spec.vocab,
+            "parallelism": "replicas x%d (independent sequences, no collective)" % world,
+            "l2": "inputs larger than L2: %.0f MB of distinct K/V, q and logits per step" % (step_bytes / 1e6),
+            "timing": "CUDA graphs replayed on one stream, CUDA events, max over ranks"}
 
 
 def run_reference(args):
+    """The CPU oracle as the timed arm: whole steps whenever the run fits a few minutes, a stated sample of layers
+    per step (and "extrapolated": true) otherwise."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     spec = synth.SPECS[args.workload]
     tb = synth.make_trees(spec)
     logits = synth.make_logits(spec, tb)
-    per_step_layers = max(1, oracle_sample_layers(spec, tb) // max(1, args.steps + args.warmup))
+    # one layer first, to know what a layer costs on this host; then as many layers per step as about 150 s allow
+    t0 = time.perf_counter()
+    time_oracle_step(spec, tb, logits, 1)
+    per_layer = max(1e-4, (time.perf_counter() - t0))
+    n_runs = max(1, args.steps + args.warmup)
+    per_step_layers = max(1, min(spec.n_layers, int(150.0 / n_runs / per_layer)))
     for _ in range(args.warmup):
         time_oracle_step(spec, tb, logits, per_step_layers)
-    times, threads, desc = [], 1, ""
+    times, threads, desc, extrapolated = [], 1, "", False
     for _ in range(args.steps):
-        t, threads, desc = time_oracle_step(spec, tb, logits, per_step_layers)
+        t, threads, desc, extrapolated = time_oracle_step(spec, tb, logits, per_step_layers)
         times.append(t)
     sec = sum(times) / len(times)
     val = 1.0 / sec
+    cfg = config_of(args, spec, tb, 1)
+    cfg["timing"] = "CPU oracle on the host cores, perf_counter"
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "note": "CPU oracle, host cores only"},
+            "config": cfg, "extrapolated": extrapolated,
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -245,7 +276,13 @@ def run_falcon(args):
     def i32(a):
         return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
 
-    node_off, parent, token, prefix = i32(tb.node_off), i32(tb.parent), i32(tb.token), i32(tb.prefix_len)
+    # the tree arrays live in one device buffer (node_off, parent, token, prefix_len), which the end-to-end leg
+    # refreshes from pinned host memory every step
+    tree_host = torch.from_numpy(np.concatenate([tb.node_off, tb.parent, tb.token, tb.prefix_len]).astype(np.int32)
+                                 ).pin_memory()
+    tree_dev = tree_host.to(dev)
+    o1, o2, o3 = B + 1, B + 1 + N, B + 1 + 2 * N
+    node_off, parent, token, prefix = tree_dev[:o1], tree_dev[o1:o2], tree_dev[o2:o3], tree_dev[o3:]
     status = torch.zeros(B, dtype=torch.int32, device=dev)
     host_prefix = np.ascontiguousarray(tb.prefix_len, dtype=np.int32)   # the caller knows these: no device round trip
     host_node_off = np.ascontiguousarray(tb.node_off, dtype=np.int32)
@@ -273,9 +310,6 @@ def run_falcon(args):
     q_all.copy_(q_host)
     logits_host = torch.from_numpy(logits_h).pin_memory()
     logits = logits_host.to(dev)
-    tree_host = torch.from_numpy(np.concatenate([tb.node_off, tb.parent, tb.token, tb.prefix_len]).astype(np.int32)
-                                 ).pin_memory()
-    tree_dev = torch.empty_like(tree_host, device=dev)
 
     g = torch.zeros(N, dtype=torch.int32, device=dev)
     path = torch.zeros((B, 128), dtype=torch.int32, device=dev)
@@ -288,10 +322,12 @@ def run_falcon(args):
     vptr = torch.tensor([cache[l, 1].data_ptr() for l in range(NL)], dtype=torch.int64, device=dev)
     strides = tuple(int(s) for s in cache[0, 0].stride()[:3])
 
-    # the prefix rows were written in earlier steps: the kernel may ask for them while the previous launch drains
-    # ... and each call names the next layer's caches, whose prefix rows it may have brought into L2
+    # The prefix rows were written in earlier steps: from the second layer on the kernel may ask for them while
+    # the previous launch drains (the first layer follows the compaction of the previous step, which writes the
+    # rows the new prefix ends with, so it makes no such promise), and each call names the next layer's caches,
+    # whose prefix rows it may have brought into L2.
     attn = [binding.attn_args(tree, Hq, Hkv, D, scale, q_all[l], out_all[l], cache[l, 0], cache[l, 1], strides, s_cap,
-                              flags=binding.ATTN_PREFIX_STABLE, kernel=ATTN_KERNELS[args.attn_kernel],
+                              flags=binding.ATTN_PREFIX_STABLE if l > 0 else 0, kernel=ATTN_KERNELS[args.attn_kernel],
                               next_k_cache=cache[l + 1, 0] if l + 1 < NL and not args.no_next_hint else None,
                               next_v_cache=cache[l + 1, 1] if l + 1 < NL and not args.no_next_hint else None)
             for l in range(NL)]
@@ -388,7 +424,8 @@ def run_falcon(args):
         pass
     peak = float(peaks.get("hbm_gbs", 6650.0))
     achieved = a_bytes / (per_launch_us * 1e-6) / 1e9
-    traffic = recorded_traffic(args.workload)
+    kernel_name = {1: "simt", 2: "tc", 3: "tck"}.get(ctx.falcon_tree_attn_kernel(attn[-1]), "?")
+    traffic = recorded_traffic(args.workload, kernel_name)
 
     if rank != 0:
         if world > 1:
@@ -401,21 +438,19 @@ def run_falcon(args):
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         sl = oracle_sample_layers(spec, tb)
-        sec, threads, desc = time_oracle_step(spec, tb, logits_h, sl)
-        cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+        sec, threads, desc, extrapolated = time_oracle_step(spec, tb, logits_h, sl)
+        sec1, _, desc1, _ = time_oracle_step(spec, tb, logits_h, max(1, sl // 8), n_threads=1)
+        cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
+               "extrapolated": extrapolated,
+               "single_thread": {"value": 1.0 / sec1, "unit": UNIT, "cores": 1, "sample": desc1}}
 
-    step_bytes = NL * a_bytes + accept_bytes(spec, tb)
     line = {
         "metric": METRIC, "value": fdist.whole_job_rate(1.0, world, ms_per_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, "batch": B, "n_layers": NL, "n_q_heads": Hq, "n_kv_heads": Hkv,
-                   "head_dim": D, "prefix_len": tb.prefix_len.tolist(), "tree_nodes": np.diff(tb.node_off).tolist(),
-                   "vocab": spec.vocab, "parallelism": "replicas x%d (independent sequences, no collective)" % world,
-                   "l2": "inputs larger than L2: %.0f MB of distinct K/V, q and logits per step" % (step_bytes / 1e6),
-                   "timing": "CUDA graphs replayed on one stream, CUDA events, max over ranks"},
+        "config": config_of(args, spec, tb, world),
         "us_per_layer": per_launch_us,
-        "roofline": {"bound": "hbm", "kernel": "falcon_tree_attn", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "roofline": {"bound": "hbm", "kernel": "falcon_tree_attn (tree_attn_%s.cu)" % kernel_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "bytes_per_launch": a_bytes,
                      "us_per_launch": per_launch_us,
                      "peak_source": "MEASURED_PEAKS.json hbm_gbs" if peaks else "fallback 6650 GB/s"},
@@ -437,7 +472,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="v7b", choices=sorted(synth.SPECS))
+    ap.add_argument("--workload", default="v7b", choices=sorted(synth.SPECS) + ["all"],
+                    help="one of the five configurations (default: the metric's), or 'all': one JSON line each (1 GPU)")
     ap.add_argument("--impl", default="falcon", choices=["falcon", "reference"])
     ap.add_argument("--attn-kernel", default="auto", choices=sorted(ATTN_KERNELS),
                     help="which attention kernel falcon_tree_attn is asked for (auto = the library's choice)")
@@ -446,6 +482,19 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "falcon":
         args.warmup = 3
+    if args.workload == "all":
+        # every configuration in a process of its own (each holds up to a few GB of caches), one line each
+        for name in ("tiny", "v7b", "l13b", "l70b", "ragged"):
+            cmd = [sys.executable, os.path.abspath(__file__), "--workload", name, "--steps", str(args.steps), "--warmup",
+                   str(args.warmup), "--impl", args.impl, "--attn-kernel", args.attn_kernel, "--no-cpu-baseline"]
+            if args.no_next_hint:
+                cmd.append("--no-next-hint")
+            r = subprocess.run(cmd, capture_output=True, text=True)
+            sys.stdout.write(r.stdout)
+            if r.returncode:
+                sys.stderr.write(r.stderr[-2000:])
+                sys.exit(r.returncode)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -110,9 +110,15 @@ typedef struct {
  *             of sequence b holds tree node t's K/V unless k_tree/v_tree given.
  *             Base 16-byte aligned, strides multiples of 8 elements.
  * k/v_tree    optional bf16 [N, Hkv, D]: tree K/V kept outside the cache.
- * kernel      FALCON_ATTN_AUTO picks; the others force one kernel (tests).
+ * kernel      FALCON_ATTN_AUTO picks (by shape, see DESIGN notes in the sources); the others force
+ *             one kernel: _SIMT CUDA cores (any supported shape), _TC tensor cores with the query
+ *             rows on the tensor-memory lanes, _TCK tensor cores with the keys on the lanes.
+ *             The tensor-core kernels need head_dim 128, the tree's K/V in the cache and Hq/Hkv a
+ *             power of two; a forced kernel that cannot take the shape returns
+ *             FALCON_ERR_UNSUPPORTED.
  * n_splits    0 = automatic; else the number of KV splits per head (1..8 for
- *             the tensor-core kernel, 1..64 for the SIMT kernel).
+ *             the tensor-core kernels, an upper bound: _TCK lowers it when the other
+ *             splits' partial results would not fit its shared memory; 1..64 for _SIMT).
  * flags       FALCON_ATTN_PREFIX_STABLE: the caller states that rows [0, L_b) of
  *             k/v_cache were last written by work that had COMPLETED before the
  *             kernel that precedes this call on the stream started (true for a
@@ -152,6 +158,10 @@ typedef struct {
 } falcon_attn_args;
 
 int falcon_tree_attn(falcon_ctx* ctx, const falcon_attn_args* args, void* stream);
+/* Which kernel falcon_tree_attn would run for these arguments (FALCON_ATTN_SIMT, _TC or _TCK; for
+ * args->kernel == FALCON_ATTN_AUTO the library's choice by shape), or -1 if it would refuse them.
+ * Launches nothing; the device pointers are not dereferenced. */
+int falcon_tree_attn_kernel(falcon_ctx* ctx, const falcon_attn_args* args);
 
 /* ---------------------------------------------------------------------------
  * falcon_tree_accept - greedy acceptance (Section 4.1 temperature 0; Section 3.4

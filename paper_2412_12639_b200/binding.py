@@ -90,6 +90,8 @@ def load_library():
         fn = getattr(lib, name)
         fn.argtypes = [C.c_void_p, C.POINTER(argt), C.c_void_p]
         fn.restype = C.c_int
+    lib.falcon_tree_attn_kernel.argtypes = [C.c_void_p, C.POINTER(AttnArgs)]
+    lib.falcon_tree_attn_kernel.restype = C.c_int
     lib.falcon_tree_accept_static.argtypes = [C.POINTER(AcceptArgs), C.c_void_p]
     lib.falcon_tree_accept_static.restype = C.c_int
     _lib = lib
@@ -179,6 +181,10 @@ class Context:
         if check:
             self._check(rc, "falcon_tree_attn")
         return rc
+
+    def falcon_tree_attn_kernel(self, args: AttnArgs) -> int:
+        """The kernel (ATTN_SIMT / ATTN_TC / ATTN_TCK) falcon_tree_attn would run for `args`, -1 if it would refuse."""
+        return int(self._lib.falcon_tree_attn_kernel(self._h, C.byref(args)))
 
     def falcon_tree_accept(self, args: AcceptArgs, stream=None, check: bool = True) -> int:
         rc = self._lib.falcon_tree_accept(self._h, C.byref(args), _stream(stream))

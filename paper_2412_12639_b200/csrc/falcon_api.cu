@@ -114,7 +114,9 @@ int falcon_tree_validate_host(const int32_t* parent, int32_t T) {
   return FALCON_OK;
 }
 
-int falcon_tree_attn(falcon_ctx* ctx, const falcon_attn_args* a, void* stream) {
+// Argument checks of falcon_tree_attn and the kernel it dispatches to; *kernel is one of
+// FALCON_ATTN_SIMT / _TC / _TCK on success.
+static int attn_plan(falcon_ctx* ctx, const falcon_attn_args* a, int* kernel) {
   if (!ctx || !a) return FALCON_ERR_INVALID_ARG;
   int rc = check_tree_desc(a->tree, false);
   if (rc) return rc;
@@ -131,24 +133,44 @@ int falcon_tree_attn(falcon_ctx* ctx, const falcon_attn_args* a, void* stream) {
   if (align & 15) return FALCON_ERR_INVALID_ARG;
   if (a->n_splits < 0 || a->n_splits > 64) return FALCON_ERR_INVALID_ARG;
   if (!(a->sm_scale == a->sm_scale)) return FALCON_ERR_INVALID_ARG;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
   switch (a->kernel) {
     case FALCON_ATTN_SIMT:
-      return launch_tree_attn_simt(ctx, *a, s);
+      *kernel = FALCON_ATTN_SIMT;
+      return FALCON_OK;
     case FALCON_ATTN_TC:
       if (!tree_attn_tc_supports(ctx, *a)) return FALCON_ERR_UNSUPPORTED;
-      return launch_tree_attn_tc(ctx, *a, s);
+      *kernel = FALCON_ATTN_TC;
+      return FALCON_OK;
     case FALCON_ATTN_TCK:
       if (!tree_attn_tck_supports(ctx, *a)) return FALCON_ERR_UNSUPPORTED;
-      return launch_tree_attn_tck(ctx, *a, s);
+      *kernel = FALCON_ATTN_TCK;
+      return FALCON_OK;
     case FALCON_ATTN_AUTO:
       if (tree_attn_tck_supports(ctx, *a) && (tree_attn_tck_preferred(ctx, *a) || !tree_attn_tc_supports(ctx, *a)))
-        return launch_tree_attn_tck(ctx, *a, s);
-      if (tree_attn_tc_supports(ctx, *a)) return launch_tree_attn_tc(ctx, *a, s);
-      return launch_tree_attn_simt(ctx, *a, s);
+        *kernel = FALCON_ATTN_TCK;
+      else if (tree_attn_tc_supports(ctx, *a))
+        *kernel = FALCON_ATTN_TC;
+      else
+        *kernel = FALCON_ATTN_SIMT;
+      return FALCON_OK;
     default:
       return FALCON_ERR_INVALID_ARG;
   }
+}
+
+int falcon_tree_attn_kernel(falcon_ctx* ctx, const falcon_attn_args* a) {
+  int kernel = -1;
+  return attn_plan(ctx, a, &kernel) == FALCON_OK ? kernel : -1;
+}
+
+int falcon_tree_attn(falcon_ctx* ctx, const falcon_attn_args* a, void* stream) {
+  int kernel = -1;
+  const int rc = attn_plan(ctx, a, &kernel);
+  if (rc) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (kernel == FALCON_ATTN_TCK) return launch_tree_attn_tck(ctx, *a, s);
+  if (kernel == FALCON_ATTN_TC) return launch_tree_attn_tc(ctx, *a, s);
+  return launch_tree_attn_simt(ctx, *a, s);
 }
 
 int falcon_tree_accept(falcon_ctx* ctx, const falcon_accept_args* a, void* stream) {

@@ -39,10 +39,11 @@ def test_recorded_traffic_is_tied_to_the_kernel_source(tmp_path, monkeypatch):
     (tmp_path / "profiles" / "tree_attn_tc_v7b_ncu.md").write_text(
         "| x |\n\ndram_bytes_per_launch: 18317312\nkernel_source_sha256: %s\n" % sha)
     monkeypatch.setattr(bench, "ROOT", str(tmp_path))
-    assert bench.recorded_traffic("v7b") == 18317312
-    assert bench.recorded_traffic("l13b") is None                 # no summary for that workload
+    assert bench.recorded_traffic("v7b", "tc") == 18317312
+    assert bench.recorded_traffic("l13b", "tc") is None           # no summary for that workload
+    assert bench.recorded_traffic("v7b", "tck") is None           # nor for the other kernel
     (src_dir / "tree_attn_tc.cu").write_bytes(b"kernel v2")        # the kernel changed since the capture
-    assert bench.recorded_traffic("v7b") is None
+    assert bench.recorded_traffic("v7b", "tc") is None
 
 
 def test_reference_arm_prints_one_line_on_the_small_workload():
@@ -54,3 +55,8 @@ def test_reference_arm_prints_one_line_on_the_small_workload():
     line = json.loads(p.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["metric"] == "tree-verify steps/sec" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+    # the same description of the workload as the GPU arm prints, and whole steps (no extrapolation) when they fit
+    assert line["extrapolated"] is False and "one whole step" in line["cpu_baseline"]["sample"]
+    spec = synth.SPECS["tiny"]
+    assert line["config"]["workload"] == "tiny" and line["config"]["n_layers"] == spec.n_layers
+    assert set(line["config"]) == set(bench.config_of(type("A", (), {"workload": "tiny"})(), spec, synth.make_trees(spec), 1))
