@@ -135,7 +135,15 @@ typedef struct {
  *             and only rows [0, L_b) are touched (they must be readable).
  * ------------------------------------------------------------------------- */
 enum { FALCON_ATTN_AUTO = 0, FALCON_ATTN_SIMT = 1, FALCON_ATTN_TC = 2, FALCON_ATTN_TCK = 3 };
-enum { FALCON_ATTN_PREFIX_STABLE = 1 };
+enum {
+  FALCON_ATTN_PREFIX_STABLE = 1,
+  /* Test hook for the bounded waits of the tensor-core kernels: the first key tile of every thread
+   * block is never requested, so the wait for it runs out (about half a second), the kernel sets
+   * FALCON_DEV_TIMEOUT in tree.status, drains what is in flight and returns; the context stays
+   * usable.  Needs n_splits == 1 and kernel == FALCON_ATTN_TC or _TCK.  The keys-on-lanes kernel still
+   * delivers the rows (by its exact fallback path), the other one writes zeros. */
+  FALCON_ATTN_TEST_STALL = 1 << 30
+};
 
 typedef struct {
   falcon_tree_desc tree;

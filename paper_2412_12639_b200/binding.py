@@ -17,6 +17,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_BAD_TREE, ERR_CAPACITY, ERR_
 DEV_BAD_TREE, DEV_CAPACITY, DEV_BAD_PATH, DEV_TIMEOUT = 1, 2, 4, 8
 ATTN_AUTO, ATTN_SIMT, ATTN_TC, ATTN_TCK = 0, 1, 2, 3
 ATTN_PREFIX_STABLE = 1
+ATTN_TEST_STALL = 1 << 30
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libfalcon.so")
 

@@ -133,6 +133,9 @@ static int attn_plan(falcon_ctx* ctx, const falcon_attn_args* a, int* kernel) {
   if (align & 15) return FALCON_ERR_INVALID_ARG;
   if (a->n_splits < 0 || a->n_splits > 64) return FALCON_ERR_INVALID_ARG;
   if (!(a->sm_scale == a->sm_scale)) return FALCON_ERR_INVALID_ARG;
+  if ((a->flags & FALCON_ATTN_TEST_STALL) &&
+      (a->n_splits != 1 || (a->kernel != FALCON_ATTN_TC && a->kernel != FALCON_ATTN_TCK)))
+    return FALCON_ERR_INVALID_ARG;
   switch (a->kernel) {
     case FALCON_ATTN_SIMT:
       *kernel = FALCON_ATTN_SIMT;

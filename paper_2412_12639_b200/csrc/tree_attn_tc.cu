@@ -117,6 +117,7 @@ struct TcParams {
   // with them the first loads do not have to wait for a round trip to global memory.
   int32_t have_host;
   int32_t early_prefix;  // prefix tiles may be requested before the previous kernel has completed
+  int32_t stall_first;   // test hook: tile 0 is never requested (a bounded wait then runs out)
   int32_t h_node_off[kHostSeqs + 1];
   int32_t h_prefix[kHostSeqs];
   FALCON_TRACE_PARAMS
@@ -190,11 +191,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int ke = min(Sv, (((split + 1) * nt + n_splits - 1) / n_splits) * kBN);
         const int nm = (ke - kb + kBN - 1) / kBN;
         for (int j = 0; j < min(nm, kPrefetch) && kb + (j + 1) * kBN <= Lq; ++j) {
+          ++n_early;
+          if (j == 0 && p.stall_first) continue;
           const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
           mbar_expect_tx(bar(kBarKVFull + j), 2 * kTileBytes);
           load_kv_tile(kdst, &tm_k, bar(kBarKVFull + j), kb + j * kBN, kvh, b);
           load_kv_tile(kdst + kTileBytes, &tm_v, bar(kBarKVFull + j), kb + j * kBN, kvh, b);
-          ++n_early;
         }
       }
     }
@@ -291,6 +293,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
       const int pre = min(n_my, kPrefetch);
       for (int j = n_early; j < pre; ++j) {
+        if (j == 0 && p.stall_first) continue;
         const uint32_t kdst = smem_base + kOffKV + j * 2 * kTileBytes;
         mbar_expect_tx(bar(kBarKVFull + j), 2 * kTileBytes);
         load_kv_tile(kdst, &tm_k, bar(kBarKVFull + j), key_begin + j * kBN, kvh, b);
@@ -313,6 +316,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (warp == kWarpProducer) {
     // ================================ TMA producer (ring refills) ================================
     if (lane == 0) {
+      int issued = min(n_my, kPrefetch);
       for (int j = kPrefetch; j < n_my; ++j) {
         const int st = j % kStages, u = j / kStages;
         // Ramp: the stages not used yet are filled one by one as earlier tiles land (a deep first
@@ -330,6 +334,25 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         mbar_expect_tx(bar(kBarKVFull + st), 2 * kTileBytes);
         load_kv_tile(kdst, &tm_k, bar(kBarKVFull + st), k0, kvh, b);
         load_kv_tile(vdst, &tm_v, bar(kBarKVFull + st), k0, kvh, b);
+        issued = j + 1;
+      }
+      if (*abort_flag) {
+        // Some wait gave up.  What was asked for still arrives: stay until it has (bounded, without
+        // looking at the abort flag), so that no copy is in flight into this CTA's shared memory
+        // when it leaves.
+        auto drain = [&](uint32_t b_, uint32_t parity) {
+          for (uint32_t it = 0; it < (1u << 20); ++it) {
+            uint32_t ok;
+            asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                         : "=r"(ok)
+                         : "r"(b_), "r"(parity)
+                         : "memory");
+            if (ok) return;
+          }
+        };
+        if (n_my > 0) drain(bar(kBarQ), 0);
+        for (int j = max(0, issued - kStages); j < issued; ++j)
+          if (!(j == 0 && p.stall_first)) drain(bar(kBarKVFull + j % kStages), (j / kStages) & 1);
       }
     }
   } else if (warp == kWarpMma) {
@@ -780,6 +803,18 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     FALCON_TRACE(tid == 0, 76);
   }
   if (warp == kWarpMma) {
+    if (n_my > 0 && *abort_flag && lane == 0) {
+      // after a wait that gave up, MMAs may still be running: the last commit covers them all
+      for (uint32_t it = 0; it < (1u << 20); ++it) {
+        uint32_t ok;
+        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                     : "=r"(ok)
+                     : "r"(bar(kBarODone)), "r"(0u)
+                     : "memory");
+        if (ok) break;
+      }
+    }
+    __syncwarp();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
@@ -898,6 +933,7 @@ int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t
   p.tree_mask = a.tree_mask;
   p.have_host = 0;
   p.early_prefix = (a.flags & FALCON_ATTN_PREFIX_STABLE) ? 1 : 0;
+  p.stall_first = (a.flags & FALCON_ATTN_TEST_STALL) ? 1 : 0;
   if (a.tree.prefix_len_host && a.tree.node_off_host && B <= kHostSeqs) {
     p.have_host = 1;
     for (int i = 0; i <= B; ++i) p.h_node_off[i] = a.tree.node_off_host[i];

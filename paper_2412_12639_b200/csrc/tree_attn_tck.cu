@@ -124,6 +124,7 @@ struct TckParams {
   __nv_bfloat16* out;
   int32_t have_host;
   int32_t early_prefix;
+  int32_t stall_first;     // test hook: tile 0 is never requested (a bounded wait then runs out)
   int32_t prefetch_next;   // tm_nk / tm_nv describe the caches of the next call: bring their prefix tiles into L2
   int32_t h_node_off[kHostSeqs + 1];
   int32_t h_prefix[kHostSeqs];
@@ -366,6 +367,7 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
   };
   const uint64_t kv_policy = policy_evict_first();
   auto load_tile = [&](int j) {
+    if (j == 0 && p.stall_first) return;
     const int st = j % kStages;
     const uint32_t dst = smem_base + off_kv + st * kStageBytes;
     mbar_expect_tx(bar(kBarKVFull + st), kStageBytes);
@@ -505,7 +507,8 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
       if (!ok || *abort_flag) {
         // Some wait gave up.  The tiles asked for still arrive: stay until they have, so that no copy
         // is in flight into this CTA's shared memory when it leaves.
-        for (int j = max(0, issued - kStages); j < issued; ++j) mbar_wait_drain(bar(kBarKVFull + j % kStages), (j / kStages) & 1);
+        for (int j = max(0, issued - kStages); j < issued; ++j)
+          if (!(j == 0 && p.stall_first)) mbar_wait_drain(bar(kBarKVFull + j % kStages), (j / kStages) & 1);
       }
       if (p.prefetch_next && ok && n_my > 0 && n_my <= kStages) {
         // The caller named the caches of the next call.  Where a CTA's whole key range fits the ring
@@ -1022,6 +1025,7 @@ int launch_impl(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s, int 
   p.have_host = 0;
   p.early_prefix = (a.flags & FALCON_ATTN_PREFIX_STABLE) ? 1 : 0;
   p.prefetch_next = prefetch_next ? 1 : 0;
+  p.stall_first = (a.flags & FALCON_ATTN_TEST_STALL) ? 1 : 0;
   if (a.tree.prefix_len_host && a.tree.node_off_host && B <= kHostSeqs) {
     p.have_host = 1;
     for (int i = 0; i <= B; ++i) p.h_node_off[i] = a.tree.node_off_host[i];

@@ -759,3 +759,33 @@ def test_captured_graph_survives_a_later_call_that_needs_more_scratch():
     want_v, want_i = oracle.topm(big.cpu().numpy(), 8)
     np.testing.assert_array_equal(idx.cpu().numpy(), want_i)
     c.close()
+
+
+@pytest.mark.parametrize("tck", TC_KERNELS)
+@pytest.mark.parametrize("T", [60, 80])
+def test_attn_bounded_wait_runs_out_and_the_context_stays_usable(tck, T):
+    """The test hook FALCON_ATTN_TEST_STALL never requests a block's first key tile, so the wait for it runs out:
+    the launch must return (no hang), report FALCON_DEV_TIMEOUT in the status word, leave finite rows (the
+    keys-on-lanes kernel still delivers the right ones through its exact fallback path, the other kernel zeros),
+    and the next ordinary launch on the same context must match the oracle."""
+    rng = np.random.default_rng(4242 + T)
+    tb, q, k, v = random_case(rng, [T], [400], 2, 2, 128)
+    ref = oracle_attn(tb, 2, 2, 128, q, k, v)
+    dt = H.DevTrees(tb)
+    out, rc = H.run_attn(dt, 2, 2, 128, q, k, v, kernel=tck, n_splits=1, flags=binding.ATTN_TEST_STALL, check=False)
+    tc_or_skip(rc)
+    assert dt.status.cpu().numpy()[0] & binding.DEV_TIMEOUT
+    got = synth.bf16_bits_to_f32(out)
+    assert np.isfinite(got).all()
+    if tck == binding.ATTN_TCK:
+        H.assert_attn_close(out, ref, tb.node_off)
+    else:
+        assert not got.any()
+    dt.status.zero_()
+    out, _ = H.run_attn(dt, 2, 2, 128, q, k, v, kernel=tck)
+    H.assert_attn_close(out, ref, tb.node_off)
+    assert not dt.status.cpu().numpy().any()
+    # the hook is refused where it would leave a cluster peer waiting, and on the other kernels
+    for kw in ({"n_splits": 2, "kernel": tck}, {"n_splits": 1, "kernel": binding.ATTN_SIMT}, {"n_splits": 1}):
+        _, rc = H.run_attn(dt, 2, 2, 128, q, k, v, flags=binding.ATTN_TEST_STALL, check=False, **kw)
+        assert rc == binding.ERR_INVALID_ARG
