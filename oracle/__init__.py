@@ -144,3 +144,26 @@ def kv_compact(node_off, prefix_len, Hkv, D, cache, strides, s_cap, path, n_path
     if rc:
         raise ValueError("oracle_kv_compact failed: %d" % rc)
     return new_len
+
+
+def feature_gather(node_off, path, n_path, token, feat, out_rows=None, hidden=None, fill=0):
+    """Accepted tokens and features along the path: feat uint16 [N, row stride >= hidden] -> (feat_out uint16
+    [B, out_rows, hidden], tok_out int32 [B, out_rows]); rows past n_path[b] keep `fill`.  `hidden` defaults
+    to the row length of `feat`."""
+    node_off, n_path, token = _i32(node_off), _i32(n_path), _i32(token)
+    path = np.ascontiguousarray(path, dtype=np.int32)
+    feat = np.ascontiguousarray(feat)
+    assert feat.dtype == np.uint16 and feat.ndim == 2
+    B = len(n_path)
+    hidden = feat.shape[1] if hidden is None else hidden
+    stride = feat.shape[1]
+    out_rows = path.shape[1] if out_rows is None else out_rows
+    feat_out = np.full((B, out_rows, hidden), fill, dtype=np.uint16)
+    tok_out = np.full((B, out_rows), fill, dtype=np.int32)
+    rc = lib().oracle_feature_gather(
+        C.c_int32(B), _p(node_off, C.c_int32), _p(path, C.c_int32), C.c_int32(path.shape[1]), _p(n_path, C.c_int32),
+        _p(token, C.c_int32), _p(feat, C.c_uint16), C.c_int32(hidden), C.c_int64(stride), C.c_int32(out_rows),
+        _p(feat_out, C.c_uint16), _p(tok_out, C.c_int32))
+    if rc:
+        raise ValueError("oracle_feature_gather failed: %d" % rc)
+    return feat_out, tok_out

@@ -398,4 +398,27 @@ int oracle_kv_compact(int32_t B, const int32_t* node_off, const int32_t* prefix_
   return 0;
 }
 
+// Accepted tokens and their features (Section 3.4: "record the accepted tokens and their
+// corresponding features for the subsequent drafting phase"): for every node on the accepted
+// path, in path order, its drafted token and its row of the [N, hidden] feature matrix (16-bit
+// elements, copied bit for bit).  feat_out is [B, out_rows, hidden], tok_out [B, out_rows]; only
+// the first n_path[b] rows of a sequence are written.
+int oracle_feature_gather(int32_t B, const int32_t* node_off, const int32_t* path, int32_t path_stride,
+                          const int32_t* n_path, const int32_t* token, const uint16_t* feat, int32_t hidden,
+                          int64_t feat_stride, int32_t out_rows, uint16_t* feat_out, int32_t* tok_out) {
+  for (int32_t b = 0; b < B; ++b) {
+    const int32_t T = node_off[b + 1] - node_off[b];
+    if (n_path[b] < 1 || n_path[b] > T || n_path[b] > out_rows) return 5;
+    for (int32_t j = 0; j < n_path[b]; ++j) {
+      const int32_t t = path[static_cast<int64_t>(b) * path_stride + j];
+      if (t < 0 || t >= T) return 4;
+      const int64_t node = node_off[b] + t;
+      tok_out[static_cast<int64_t>(b) * out_rows + j] = token[node];
+      for (int32_t c = 0; c < hidden; ++c)
+        feat_out[(static_cast<int64_t>(b) * out_rows + j) * hidden + c] = feat[node * feat_stride + c];
+    }
+  }
+  return 0;
+}
+
 }  // extern "C"

@@ -578,3 +578,48 @@ def test_topm_respects_row_stride_and_permutations():
     val2, idx2 = oracle.topm(shuffled, m, vocab=V)
     np.testing.assert_array_equal(val, val2)                   # the values are a property of the multiset
     np.testing.assert_array_equal(perm[idx2], idx)             # distinct values almost surely: indices map back
+
+
+# ------------------------------------------------------------ feature gather
+def test_feature_gather_hand_worked():
+    case = GOLD["feature_gather_basic"]
+    T, Hd = len(case["parent"]), case["hidden"]
+    feat = np.array([[10 * i + c for c in range(Hd)] for i in range(T)], np.uint16)
+    path = np.full((1, 8), -1, np.int32)
+    path[0, :3] = case["path"]
+    fo, to = oracle.feature_gather([0, T], path, [case["n_path"]], case["token"], feat, fill=777)
+    np.testing.assert_array_equal(to[0, :3], case["expected_tokens"])
+    np.testing.assert_array_equal(fo[0, :3], np.array(case["expected_features"], np.uint16))
+    assert (to[0, 3:] == 777).all() and (fo[0, 3:] == 777).all()        # rows past the path are not touched
+
+
+def test_feature_gather_equals_fancy_indexing_on_random_batches():
+    rng = np.random.default_rng(91)
+    for _ in range(20):
+        B = int(rng.integers(1, 5))
+        sizes = [int(rng.integers(1, 129)) for _ in range(B)]
+        node_off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+        N, Hd = int(node_off[-1]), int(rng.choice([8, 40, 128]))
+        feat = rng.integers(0, 65536, size=(N, Hd + 8), dtype=np.uint16)       # row stride wider than hidden
+        token = rng.integers(0, 32000, size=N).astype(np.int32)
+        path = np.full((B, 128), -1, np.int32)
+        n_path = np.zeros(B, np.int32)
+        for b, T in enumerate(sizes):
+            n = int(rng.integers(1, T + 1))
+            path[b, :n] = np.sort(rng.choice(T, size=n, replace=False))     # any increasing node list will do here
+            n_path[b] = n
+        fo, to = oracle.feature_gather(node_off, path, n_path, token, feat, hidden=Hd, fill=9)
+        for b in range(B):
+            idx = node_off[b] + path[b, :n_path[b]]
+            np.testing.assert_array_equal(fo[b, :n_path[b]], feat[idx, :Hd])
+            np.testing.assert_array_equal(to[b, :n_path[b]], token[idx])
+            assert (fo[b, n_path[b]:] == 9).all() and (to[b, n_path[b]:] == 9).all()
+
+
+def test_feature_gather_rejects_bad_paths():
+    feat = np.zeros((4, 8), np.uint16)
+    path = np.array([[0, 7, -1, -1]], np.int32)                                # node 7 is outside a tree of 4
+    with pytest.raises(ValueError):
+        oracle.feature_gather([0, 4], path, [2], [1, 2, 3, 4], feat)
+    with pytest.raises(ValueError):
+        oracle.feature_gather([0, 4], np.array([[0, 1, 2, 3]], np.int32), [5], [1, 2, 3, 4], feat)
