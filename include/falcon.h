@@ -254,6 +254,37 @@ int falcon_topm(falcon_ctx* ctx, const falcon_topm_args* args, void* stream);
 int falcon_tree_accept_static(const falcon_accept_args* args, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * falcon_feature_gather - the accepted tokens and their features (Section 3.4: after
+ * verification "we record the accepted tokens and their corresponding features for the
+ * subsequent drafting phase": the drafter's next input is the target model's hidden state
+ * of every accepted node together with its token, Section 3.1).
+ *
+ *   tokens_out[b, j]      = token[node_off[b] + path[b][j]]
+ *   features_out[b, j, :] = features[node_off[b] + path[b][j], 0 .. hidden-1]    j < n_path[b]
+ * Rows j >= n_path[b] of the outputs are not written.  Features are 16-bit elements
+ * (bf16), copied bit for bit.  A path entry outside the tree sets FALCON_DEV_BAD_PATH
+ * and leaves that sequence's outputs alone.
+ *
+ *   features      [N, feat_stride], feat_stride >= hidden, both multiples of 8, 16-byte aligned
+ *   features_out  [B, out_rows, hidden], tokens_out [B, out_rows], out_rows >= max_tree
+ * The same work can ride on the compaction launch: see falcon_compact_args.gather.
+ * ------------------------------------------------------------------------- */
+typedef struct {
+  falcon_tree_desc tree;  /* token is read                                            */
+  int32_t hidden;
+  int64_t feat_stride;
+  const void* features;
+  const int32_t* path;    /* [B, path_stride] from falcon_tree_accept                 */
+  int32_t path_stride;
+  const int32_t* n_path;  /* [B]                                                      */
+  int32_t out_rows;
+  void* features_out;
+  int32_t* tokens_out;
+} falcon_gather_args;
+
+int falcon_feature_gather(falcon_ctx* ctx, const falcon_gather_args* args, void* stream);
+
+/* ---------------------------------------------------------------------------
  * falcon_kv_compact - keep the accepted path's K/V (Section 3.4: "record the
  * accepted tokens and their corresponding features for the subsequent drafting
  * phase", in its KV-cache form), all layers in one launch.
@@ -267,7 +298,7 @@ int falcon_tree_accept_static(const falcon_accept_args* args, void* stream);
  * modified.
  * ------------------------------------------------------------------------- */
 typedef struct {
-  falcon_tree_desc tree;  /* token unused                                             */
+  falcon_tree_desc tree;  /* token unused (read only when `gather` is given)          */
   int32_t n_layers, n_kv_heads, head_dim;
   void* const* k_cache_layers; /* device array [n_layers] of cache base pointers      */
   void* const* v_cache_layers;
@@ -279,6 +310,9 @@ typedef struct {
   int32_t path_stride;
   const int32_t* n_path;  /* [B]                                                      */
   int32_t* new_len;       /* [B]                                                      */
+  const falcon_gather_args* gather; /* optional HOST pointer: also record the accepted tokens and features in
+                                       this launch (its features / outputs are used; tree, path and n_path
+                                       are the compaction's, which must describe the same batch)         */
 } falcon_compact_args;
 
 int falcon_kv_compact(falcon_ctx* ctx, const falcon_compact_args* args, void* stream);

@@ -56,12 +56,19 @@ class TopmArgs(C.Structure):
                 ("m", C.c_int32), ("top_val", C.c_void_p), ("top_idx", C.c_void_p)]
 
 
+class GatherArgs(C.Structure):
+    _fields_ = [("tree", TreeDesc), ("hidden", C.c_int32), ("feat_stride", C.c_int64), ("features", C.c_void_p),
+                ("path", C.c_void_p), ("path_stride", C.c_int32), ("n_path", C.c_void_p), ("out_rows", C.c_int32),
+                ("features_out", C.c_void_p), ("tokens_out", C.c_void_p)]
+
+
 class CompactArgs(C.Structure):
     _fields_ = [("tree", TreeDesc), ("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("k_cache_layers", C.c_void_p), ("v_cache_layers", C.c_void_p), ("kv_stride_b", C.c_int64),
                 ("kv_stride_h", C.c_int64), ("kv_stride_s", C.c_int64), ("s_cap", C.c_int32),
                 ("k_tree_layers", C.c_void_p), ("v_tree_layers", C.c_void_p), ("path", C.c_void_p),
-                ("path_stride", C.c_int32), ("n_path", C.c_void_p), ("new_len", C.c_void_p)]
+                ("path_stride", C.c_int32), ("n_path", C.c_void_p), ("new_len", C.c_void_p),
+                ("gather", C.POINTER(GatherArgs))]
 
 
 _lib = None
@@ -87,7 +94,8 @@ def load_library():
     lib.falcon_tree_validate_host.argtypes = [C.c_void_p, C.c_int32]
     lib.falcon_tree_validate_host.restype = C.c_int
     for name, argt in (("falcon_tree_attn", AttnArgs), ("falcon_tree_accept", AcceptArgs),
-                       ("falcon_kv_compact", CompactArgs), ("falcon_topm", TopmArgs)):
+                       ("falcon_kv_compact", CompactArgs), ("falcon_topm", TopmArgs),
+                       ("falcon_feature_gather", GatherArgs)):
         fn = getattr(lib, name)
         fn.argtypes = [C.c_void_p, C.POINTER(argt), C.c_void_p]
         fn.restype = C.c_int
@@ -199,6 +207,12 @@ class Context:
             self._check(rc, "falcon_topm")
         return rc
 
+    def falcon_feature_gather(self, args: GatherArgs, stream=None, check: bool = True) -> int:
+        rc = self._lib.falcon_feature_gather(self._h, C.byref(args), _stream(stream))
+        if check:
+            self._check(rc, "falcon_feature_gather")
+        return rc
+
     def falcon_kv_compact(self, args: CompactArgs, stream=None, check: bool = True) -> int:
         rc = self._lib.falcon_kv_compact(self._h, C.byref(args), _stream(stream))
         if check:
@@ -226,8 +240,18 @@ def topm_args(n_rows, vocab, logits, logits_stride, m, top_val, top_idx) -> Topm
     return TopmArgs(n_rows, vocab, logits_stride, _ptr(logits), m, _ptr(top_val), _ptr(top_idx))
 
 
+def gather_args(tree: TreeDesc, hidden, features, feat_stride, path, path_stride, n_path, out_rows, features_out,
+                tokens_out) -> GatherArgs:
+    return GatherArgs(tree, hidden, feat_stride, _ptr(features), _ptr(path), path_stride, _ptr(n_path), out_rows,
+                      _ptr(features_out), _ptr(tokens_out))
+
+
 def compact_args(tree: TreeDesc, n_layers, n_kv_heads, head_dim, k_cache_layers, v_cache_layers, strides, s_cap,
-                 path, path_stride, n_path, new_len, k_tree_layers=None, v_tree_layers=None) -> CompactArgs:
+                 path, path_stride, n_path, new_len, k_tree_layers=None, v_tree_layers=None,
+                 gather: Optional[GatherArgs] = None) -> CompactArgs:
+    """gather: record the accepted tokens and features in the same launch (the caller keeps `gather` alive
+    until the call has returned)."""
     return CompactArgs(tree, n_layers, n_kv_heads, head_dim, _ptr(k_cache_layers), _ptr(v_cache_layers),
                        strides[0], strides[1], strides[2], s_cap, _ptr(k_tree_layers), _ptr(v_tree_layers),
-                       _ptr(path), path_stride, _ptr(n_path), _ptr(new_len))
+                       _ptr(path), path_stride, _ptr(n_path), _ptr(new_len),
+                       C.pointer(gather) if gather is not None else None)

@@ -45,6 +45,8 @@ int check_tree_desc(const falcon_tree_desc& t, bool need_token);
 // launchers (one per kernel file)
 int launch_tree_accept(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_t s);
 int launch_kv_compact(falcon_ctx* ctx, const falcon_compact_args& a, cudaStream_t s);
+int launch_feature_gather(falcon_ctx* ctx, const falcon_gather_args& a, cudaStream_t s);
+int check_gather_args(const falcon_gather_args& g, int max_tree);
 int launch_tree_topm(falcon_ctx* ctx, const falcon_topm_args& a, cudaStream_t s);
 int launch_tree_attn_simt(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s);
 int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s);

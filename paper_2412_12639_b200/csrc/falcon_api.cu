@@ -208,7 +208,22 @@ int falcon_kv_compact(falcon_ctx* ctx, const falcon_compact_args* a, void* strea
   if (a->kv_stride_s < a->head_dim || a->kv_stride_h < 0 || a->kv_stride_b < 0) return FALCON_ERR_INVALID_ARG;
   if ((a->kv_stride_s | a->kv_stride_h | a->kv_stride_b) & 7) return FALCON_ERR_INVALID_ARG;
   if (a->path_stride < a->tree.max_tree) return FALCON_ERR_INVALID_ARG;
+  if (a->gather) {
+    if (!a->tree.token) return FALCON_ERR_INVALID_ARG;
+    rc = check_gather_args(*a->gather, a->tree.max_tree);
+    if (rc) return rc;
+  }
   return launch_kv_compact(ctx, *a, static_cast<cudaStream_t>(stream));
+}
+
+int falcon_feature_gather(falcon_ctx* ctx, const falcon_gather_args* a, void* stream) {
+  if (!ctx || !a) return FALCON_ERR_INVALID_ARG;
+  int rc = check_tree_desc(a->tree, true);
+  if (rc) return rc;
+  if (!a->path || !a->n_path || a->path_stride < a->tree.max_tree) return FALCON_ERR_INVALID_ARG;
+  rc = check_gather_args(*a, a->tree.max_tree);
+  if (rc) return rc;
+  return launch_feature_gather(ctx, *a, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

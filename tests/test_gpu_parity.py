@@ -789,3 +789,102 @@ def test_attn_bounded_wait_runs_out_and_the_context_stays_usable(tck, T):
     for kw in ({"n_splits": 2, "kernel": tck}, {"n_splits": 1, "kernel": binding.ATTN_SIMT}, {"n_splits": 1}):
         _, rc = H.run_attn(dt, 2, 2, 128, q, k, v, flags=binding.ATTN_TEST_STALL, check=False, **kw)
         assert rc == binding.ERR_INVALID_ARG
+
+
+# ------------------------------------------------- accepted tokens and features
+def _gather_case(rng, sizes, hidden, stride_pad=0):
+    tb = H.make_trees(sizes, [0] * len(sizes), rng, vocab=32000)
+    N, B = tb.total_nodes, tb.batch
+    feat = rng.integers(0, 65536, size=(N, hidden + stride_pad), dtype=np.uint16)
+    path = np.full((B, 128), -1, np.int32)
+    n_path = np.zeros(B, np.int32)
+    for b, T in enumerate(sizes):                           # a real root-to-node chain of each tree
+        node = int(rng.integers(0, T))
+        chain = oracle.ancestors(tb.parent[tb.node_off[b]:tb.node_off[b + 1]], node)
+        chain = sorted(chain)
+        path[b, :len(chain)] = chain
+        n_path[b] = len(chain)
+    return tb, feat, path, n_path
+
+
+@pytest.mark.parametrize("sizes,hidden,pad", [([6], 8, 0), ([60], 4096, 0), ([80, 1, 33], 5120, 8),
+                                              ([128] * 3, 1024, 0), ([20, 80, 47, 64, 33, 21, 77, 50], 4096, 0)])
+def test_feature_gather_bit_exact(sizes, hidden, pad):
+    rng = np.random.default_rng(hidden + len(sizes))
+    tb, feat, path, n_path = _gather_case(rng, sizes, hidden, pad)
+    f_ref, t_ref = oracle.feature_gather(tb.node_off, path, n_path, tb.token, feat, hidden=hidden, fill=0x7777)
+    dt = H.DevTrees(tb)
+    fd = torch.from_numpy(feat.view(np.int16)).cuda()
+    pd, nd = H.dev_i32(path), H.dev_i32(n_path)
+    fo = torch.full((tb.batch, 128, hidden), 0x7777, dtype=torch.int16, device="cuda")
+    to = torch.full((tb.batch, 128), 0x7777, dtype=torch.int32, device="cuda")
+    a = binding.gather_args(dt.desc(), hidden, fd, feat.shape[1], pd, 128, nd, 128, fo, to)
+    H.ctx().falcon_feature_gather(a)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(fo.cpu().numpy().view(np.uint16), f_ref)      # rows past the path untouched too
+    np.testing.assert_array_equal(to.cpu().numpy(), t_ref)
+    assert not dt.status.cpu().numpy().any()
+
+
+def test_feature_gather_rides_on_the_compaction_launch():
+    """falcon_kv_compact with `gather`: one launch compacts the caches and records the accepted tokens and features;
+    both results equal the oracle's, bit for bit."""
+    rng = np.random.default_rng(55)
+    sizes, prefs, Hkv, D, hidden = [60, 17], [100, 31], 4, 128, 4096
+    tb = H.make_trees(sizes, prefs, rng)
+    s_cap = max(p + t for p, t in zip(prefs, sizes))
+    k = [synth.normal_bf16(rng, (2, Hkv, s_cap, D)) for _ in range(3)]
+    v = [synth.normal_bf16(rng, (2, Hkv, s_cap, D)) for _ in range(3)]
+    logits = rng.standard_normal((tb.total_nodes, 50)).astype(np.float32)
+    g = oracle.argmax(logits)
+    path, n_path, _ = oracle.tree_accept(tb.node_off, tb.parent, tb.token, g)
+    feat = rng.integers(0, 65536, size=(tb.total_nodes, hidden), dtype=np.uint16)
+    f_ref, t_ref = oracle.feature_gather(tb.node_off, path, n_path, tb.token, feat, fill=0)
+    dt = H.DevTrees(tb)
+    kd, vd = [H.dev_bf16(x) for x in k], [H.dev_bf16(x) for x in v]
+    kp = torch.tensor([t.data_ptr() for t in kd], dtype=torch.int64, device="cuda")
+    vp = torch.tensor([t.data_ptr() for t in vd], dtype=torch.int64, device="cuda")
+    pd, nd = H.dev_i32(path), H.dev_i32(n_path)
+    new_len = torch.full((2,), -7, dtype=torch.int32, device="cuda")
+    fd = torch.from_numpy(feat.view(np.int16)).cuda()
+    fo = torch.zeros((2, 128, hidden), dtype=torch.int16, device="cuda")
+    to = torch.zeros((2, 128), dtype=torch.int32, device="cuda")
+    ga = binding.gather_args(dt.desc(), hidden, fd, hidden, pd, 128, nd, 128, fo, to)
+    strides = tuple(int(s) for s in kd[0].stride()[:3])
+    ca = binding.compact_args(dt.desc(), 3, Hkv, D, kp, vp, strides, s_cap, pd, 128, nd, new_len, gather=ga)
+    H.ctx().falcon_kv_compact(ca)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(fo.cpu().numpy().view(np.uint16), f_ref)
+    np.testing.assert_array_equal(to.cpu().numpy(), t_ref)
+    st = strides_of(k[0])
+    for layer in range(3):
+        for host, devt in ((k[layer], kd[layer]), (v[layer], vd[layer])):
+            ref = host.copy()
+            nl = oracle.kv_compact(tb.node_off, tb.prefix_len, Hkv, D, ref, st, s_cap, path, n_path)
+            got = H.host_bits(devt)
+            for b in range(2):
+                np.testing.assert_array_equal(got[b, :, :nl[b]], ref[b, :, :nl[b]])
+            np.testing.assert_array_equal(new_len.cpu().numpy(), nl)
+    assert not dt.status.cpu().numpy().any()
+
+
+def test_feature_gather_bad_path_sets_status_and_writes_nothing():
+    rng = np.random.default_rng(56)
+    tb, feat, path, n_path = _gather_case(rng, [10, 12], 64)
+    path[0, 1] = 11                                         # outside sequence 0's tree of 10 nodes
+    n_path[0] = max(2, n_path[0])
+    dt = H.DevTrees(tb)
+    fd = torch.from_numpy(feat.view(np.int16)).cuda()
+    fo = torch.full((2, 128, 64), 0x1111, dtype=torch.int16, device="cuda")
+    to = torch.full((2, 128), -5, dtype=torch.int32, device="cuda")
+    a = binding.gather_args(dt.desc(), 64, fd, 64, H.dev_i32(path), 128, H.dev_i32(n_path), 128, fo, to)
+    H.ctx().falcon_feature_gather(a)
+    torch.cuda.synchronize()
+    st = dt.status.cpu().numpy()
+    assert st[0] & binding.DEV_BAD_PATH and st[1] == 0
+    assert (to.cpu().numpy()[0] == -5).all() and (fo.cpu().numpy()[0] == 0x1111).all()
+    f_ref, t_ref = oracle.feature_gather(tb.node_off[1:] - tb.node_off[1], path[1:], n_path[1:], tb.token[10:], feat[10:])
+    np.testing.assert_array_equal(to.cpu().numpy()[1, :n_path[1]], t_ref[0, :n_path[1]])
+    # bad arguments are refused on the host
+    bad = binding.gather_args(dt.desc(), 60, fd, 64, H.dev_i32(path), 128, H.dev_i32(n_path), 128, fo, to)
+    assert H.ctx().falcon_feature_gather(bad, check=False) == binding.ERR_INVALID_ARG
