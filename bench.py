@@ -244,7 +244,7 @@ def time_topm(ctx, binding, torch, dev, stream, logits_h, peak, m=20, copies=20,
 
 
 # --------------------------------------------------------------------------- GPU arm
-ATTN_KERNELS = {"auto": 0, "simt": 1, "tc": 2, "tck": 3}   # falcon.h FALCON_ATTN_*
+ATTN_KERNELS = {"auto": 0, "simt": 1, "tc": 2, "tck": 3, "warp": 4}   # falcon.h FALCON_ATTN_*
 
 
 def run_falcon(args):
@@ -424,7 +424,7 @@ def run_falcon(args):
         pass
     peak = float(peaks.get("hbm_gbs", 6650.0))
     achieved = a_bytes / (per_launch_us * 1e-6) / 1e9
-    kernel_name = {1: "simt", 2: "tc", 3: "tck"}.get(ctx.falcon_tree_attn_kernel(attn[-1]), "?")
+    kernel_name = {1: "simt", 2: "tc", 3: "tck", 4: "warp"}.get(ctx.falcon_tree_attn_kernel(attn[-1]), "?")
     traffic = recorded_traffic(args.workload, kernel_name)
 
     if rank != 0:

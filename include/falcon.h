@@ -111,8 +111,10 @@ typedef struct {
  *             Base 16-byte aligned, strides multiples of 8 elements.
  * k/v_tree    optional bf16 [N, Hkv, D]: tree K/V kept outside the cache.
  * kernel      FALCON_ATTN_AUTO picks (by shape, see DESIGN notes in the sources); the others force
- *             one kernel: _SIMT CUDA cores (any supported shape), _TC tensor cores with the query
- *             rows on the tensor-memory lanes, _TCK tensor cores with the keys on the lanes.
+ *             one kernel: _SIMT CUDA cores (any supported shape), _WARP CUDA cores with one warp
+ *             per query row (at most 1024 keys per sequence; the small-problem kernel), _TC tensor
+ *             cores with the query rows on the tensor-memory lanes, _TCK tensor cores with the
+ *             keys on the lanes.
  *             The tensor-core kernels need head_dim 128, the tree's K/V in the cache and Hq/Hkv a
  *             power of two; a forced kernel that cannot take the shape returns
  *             FALCON_ERR_UNSUPPORTED.
@@ -134,7 +136,7 @@ typedef struct {
  *             layer's tail and the launch gap.  A hint only: results never depend on it,
  *             and only rows [0, L_b) are touched (they must be readable).
  * ------------------------------------------------------------------------- */
-enum { FALCON_ATTN_AUTO = 0, FALCON_ATTN_SIMT = 1, FALCON_ATTN_TC = 2, FALCON_ATTN_TCK = 3 };
+enum { FALCON_ATTN_AUTO = 0, FALCON_ATTN_SIMT = 1, FALCON_ATTN_TC = 2, FALCON_ATTN_TCK = 3, FALCON_ATTN_WARP = 4 };
 enum {
   FALCON_ATTN_PREFIX_STABLE = 1,
   /* Test hook for the bounded waits of the tensor-core kernels: the first key tile of every thread
@@ -166,7 +168,7 @@ typedef struct {
 } falcon_attn_args;
 
 int falcon_tree_attn(falcon_ctx* ctx, const falcon_attn_args* args, void* stream);
-/* Which kernel falcon_tree_attn would run for these arguments (FALCON_ATTN_SIMT, _TC or _TCK; for
+/* Which kernel falcon_tree_attn would run for these arguments (FALCON_ATTN_SIMT, _WARP, _TC or _TCK; for
  * args->kernel == FALCON_ATTN_AUTO the library's choice by shape), or -1 if it would refuse them.
  * Launches nothing; the device pointers are not dereferenced. */
 int falcon_tree_attn_kernel(falcon_ctx* ctx, const falcon_attn_args* args);

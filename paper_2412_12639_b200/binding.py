@@ -15,7 +15,7 @@ from typing import Optional
 T_MAX = 128
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_BAD_TREE, ERR_CAPACITY, ERR_TIMEOUT = range(7)
 DEV_BAD_TREE, DEV_CAPACITY, DEV_BAD_PATH, DEV_TIMEOUT = 1, 2, 4, 8
-ATTN_AUTO, ATTN_SIMT, ATTN_TC, ATTN_TCK = 0, 1, 2, 3
+ATTN_AUTO, ATTN_SIMT, ATTN_TC, ATTN_TCK, ATTN_WARP = 0, 1, 2, 3, 4
 ATTN_PREFIX_STABLE = 1
 ATTN_TEST_STALL = 1 << 30
 

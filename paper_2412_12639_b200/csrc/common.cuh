@@ -54,6 +54,8 @@ bool tree_attn_tc_supports(const falcon_ctx* ctx, const falcon_attn_args& a);
 int launch_tree_attn_tck(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s);
 bool tree_attn_tck_supports(const falcon_ctx* ctx, const falcon_attn_args& a);
 bool tree_attn_tck_preferred(const falcon_ctx* ctx, const falcon_attn_args& a);
+int launch_tree_attn_warp(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s);
+bool tree_attn_warp_supports(const falcon_ctx* ctx, const falcon_attn_args& a);
 void tree_attn_tc_release(falcon_ctx* ctx);
 
 #ifdef __CUDACC__

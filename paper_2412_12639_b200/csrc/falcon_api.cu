@@ -148,11 +148,19 @@ static int attn_plan(falcon_ctx* ctx, const falcon_attn_args* a, int* kernel) {
       if (!tree_attn_tck_supports(ctx, *a)) return FALCON_ERR_UNSUPPORTED;
       *kernel = FALCON_ATTN_TCK;
       return FALCON_OK;
+    case FALCON_ATTN_WARP:
+      if (!tree_attn_warp_supports(ctx, *a)) return FALCON_ERR_UNSUPPORTED;
+      *kernel = FALCON_ATTN_WARP;
+      return FALCON_OK;
     case FALCON_ATTN_AUTO:
+      // tensor cores where a kernel takes the shape (which of the two: by shape, measured); else one
+      // warp per query row while the scores of a row fit its shared memory; else the tiled kernel
       if (tree_attn_tck_supports(ctx, *a) && (tree_attn_tck_preferred(ctx, *a) || !tree_attn_tc_supports(ctx, *a)))
         *kernel = FALCON_ATTN_TCK;
       else if (tree_attn_tc_supports(ctx, *a))
         *kernel = FALCON_ATTN_TC;
+      else if (tree_attn_warp_supports(ctx, *a))
+        *kernel = FALCON_ATTN_WARP;
       else
         *kernel = FALCON_ATTN_SIMT;
       return FALCON_OK;
@@ -173,6 +181,7 @@ int falcon_tree_attn(falcon_ctx* ctx, const falcon_attn_args* a, void* stream) {
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (kernel == FALCON_ATTN_TCK) return launch_tree_attn_tck(ctx, *a, s);
   if (kernel == FALCON_ATTN_TC) return launch_tree_attn_tc(ctx, *a, s);
+  if (kernel == FALCON_ATTN_WARP) return launch_tree_attn_warp(ctx, *a, s);
   return launch_tree_attn_simt(ctx, *a, s);
 }
 

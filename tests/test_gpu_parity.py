@@ -14,13 +14,13 @@ import gpu_harness as H
 
 pytestmark = pytest.mark.gpu
 
-KERNELS = [binding.ATTN_SIMT, binding.ATTN_TC, binding.ATTN_TCK]
+KERNELS = [binding.ATTN_SIMT, binding.ATTN_WARP, binding.ATTN_TC, binding.ATTN_TCK]
 TC_KERNELS = [binding.ATTN_TC, binding.ATTN_TCK]      # queries / keys on the tensor-memory lanes
 
 
 def tc_or_skip(rc):
     if rc == binding.ERR_UNSUPPORTED:
-        pytest.skip("shape not taken by the tensor-core kernel")
+        pytest.skip("shape not taken by this kernel")
     assert rc == binding.OK
 
 
