@@ -65,6 +65,17 @@ def recorded_traffic(workload: str, kernel: str):
     return int(val.group(1))
 
 
+def traffic_note(workload: str, kernel: str):
+    """The one-line remark a summary may carry next to its DRAM bytes (`traffic_note: ...`), or None."""
+    import re
+    try:
+        text = open(os.path.join(ROOT, "profiles", "tree_attn_%s_%s_ncu.md" % (kernel, workload))).read()
+    except OSError:
+        return None
+    m = re.search(r"traffic_note:\s*(.+)", text)
+    return m.group(1).strip() if m else None
+
+
 # --------------------------------------------------------------------------- clocks
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
@@ -451,7 +462,9 @@ def run_falcon(args):
         "config": config_of(args, spec, tb, world),
         "us_per_layer": per_launch_us,
         "roofline": {"bound": "hbm", "kernel": "falcon_tree_attn (tree_attn_%s.cu)" % kernel_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": traffic, "bytes_per_launch": a_bytes,
+                     "frac": achieved / peak, "traffic": traffic,
+                     "traffic_note": traffic_note(args.workload, kernel_name) if traffic is not None else None,
+                     "bytes_per_launch": a_bytes,
                      "us_per_launch": per_launch_us,
                      "peak_source": "MEASURED_PEAKS.json hbm_gbs" if peaks else "fallback 6650 GB/s"},
         "e2e": {"value": fdist.whole_job_rate(e2e_steps, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
