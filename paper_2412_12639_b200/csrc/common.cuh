@@ -29,10 +29,10 @@ struct falcon_ctx {
   void* tmap_cache = nullptr;
   // Per-context launch state of the tensor-core attention kernels: whether the dynamic shared
   // memory limit has been raised on this device, and how many clusters of each size fit at once
-  // (0 = not asked yet, -1 = none).  Index 0: rows-on-lanes kernel; 1, 2: keys-on-lanes kernel
-  // (small and large query block).
-  bool attn_attr_set[3] = {false, false, false};
-  int attn_resident[3][9] = {};
+  // (0 = not asked yet, -1 = none).  Index 0: rows-on-lanes kernel; 1-3: the keys-on-lanes kernel's
+  // three variants.
+  bool attn_attr_set[4] = {false, false, false, false};
+  int attn_resident[4][9] = {};
 };
 
 namespace falcon {

@@ -54,10 +54,26 @@ using namespace tc;
 
 constexpr int kD = 128;
 constexpr int kBKMax = 128;                     // keys per tile at most = TMEM lanes (the launcher picks the tile height)
-constexpr int kColGroups = 4;                   // softmax warps per lane quadrant
-constexpr int kSmWarps = 4 * kColGroups;
-constexpr int kSmThreads = 32 * kSmWarps;       // 512
-constexpr int kThreads = 32 * (2 + kSmWarps);   // 576
+// Three variants by the number of query rows N of a unit.  A softmax thread works on chunks of kCW
+// query columns; chunk c belongs to column group c % kGroups, and a lane quadrant has one warp per
+// column group.
+//   0: N <= 64   4 groups, one chunk of 16 columns a thread             (18 warps)
+//   1: N <= 80   5 groups, one chunk of 16 columns a thread             (22 warps)
+//   2: N <= 128  4 groups, up to four chunks of 8 columns a thread, so that e.g. 96 rows spread
+//                evenly; registers do not hold all chunks at once, so they are handled in turn
+template <int kVar>
+struct Var {
+  static constexpr int kGroups = kVar == 1 ? 5 : 4;
+  static constexpr int kCW = kVar == 2 ? 8 : 16;
+  static constexpr int kPer = kVar == 2 ? 4 : 1;
+  static constexpr int kNMax = kVar == 0 ? 64 : (kVar == 1 ? 80 : 128);
+  static constexpr int kCfg = kVar == 0 ? 1 : 2;           // which Cfg (small arrays sized for 64 or 128 rows)
+  static constexpr int kSmWarps = 4 * kGroups;
+  static constexpr int kSmThreads = 32 * kSmWarps;
+  static constexpr int kThreads = 32 * (2 + kSmWarps);     // producer, MMA issuer, softmax warps
+  static constexpr int kRowsPerPass = kSmThreads / 8;      // Q rows the softmax threads load at once (8 threads a row)
+  static constexpr int kQPasses = (kNMax + kRowsPerPass - 1) / kRowsPerPass;
+};
 constexpr int kWarpProducer = 0;
 constexpr int kWarpMma = 1;
 constexpr int kWarpSm0 = 2;
@@ -82,7 +98,7 @@ enum {
   kNumBars = kBarMrg + 1
 };
 
-// kChunks = 1: up to 64 query rows per unit; kChunks = 2: up to 128.  Shared memory, from offset 0:
+// kChunks = 1: room for 64 query rows per unit; kChunks = 2: for 128.  Shared memory, from offset 0:
 // the Q block (n_rows x 256 bytes), the K/V ring (stages x tile_keys x 512 bytes), the merge area
 // (what the other splits deliver), and a block of small arrays whose layout is below.  The ring
 // takes what the rest leaves: the launcher picks the tile height and the number of stages.
@@ -295,12 +311,14 @@ __device__ void rescue_row(const TckParams& p, int b, int kvh, int node_base, in
 }
 
 // kFull: the ring is three stages of 128-key tiles (then the geometry is known at compile time).
-template <int kChunks, bool kFull>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int kVar, bool kFull>
+__global__ void __launch_bounds__(Var<kVar>::kThreads, 1)
 tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                      const __grid_constant__ CUtensorMap tm_nk, const __grid_constant__ CUtensorMap tm_nv,
                      const TckParams p) {
-  using C = Cfg<kChunks>;
+  using VT = Var<kVar>;
+  using C = Cfg<VT::kCfg>;
+  constexpr int kColGroups = VT::kGroups, kSmWarps = VT::kSmWarps, kSmThreads = VT::kSmThreads, kThreads = VT::kThreads;
   extern __shared__ __align__(1024) unsigned char smem_gen[];
   const uint32_t smem_base = smem_u32(smem_gen);
   unsigned char* small = smem_gen + p.off_small;
@@ -316,16 +334,13 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
   const uint32_t kHalfTile = static_cast<uint32_t>(BK) * 128u;   // one 64-column half of a K or V tile
   const uint32_t kTileBytes = 2u * kHalfTile, kStageBytes = 2u * kTileBytes;
   const uint32_t off_q = 0, off_kv = static_cast<uint32_t>(p.n_rows) * 256u, off_mrg = p.off_mrg, off_stage = 0;
-  const uint32_t tmem_cols = (kChunks == 1 || p.n_rows <= 64) ? 256u : 512u, col_stride = tmem_cols / 4;  // S^T(0), S^T(1), O^T
+  const uint32_t tmem_cols = (kVar == 0 || p.n_rows <= 64) ? 256u : 512u, col_stride = tmem_cols / 4;  // S^T(0), S^T(1), O^T
   auto bar = [&](int i) { return bars + 8u * static_cast<uint32_t>(i); };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n_splits = gridDim.x, split = blockIdx.x;  // cluster = all CTAs of a row of the grid
   const int kvh = blockIdx.y % p.Hkv, mtile = blockIdx.y / p.Hkv, b = blockIdx.z;
-  // A softmax thread works on chunks of kCW query columns: one chunk of 16 when there are at most 64
-  // rows, up to four chunks of 8 otherwise (chunk c goes to column group c % 4, so 80 rows spread as
-  // 24, 24, 16, 16 columns).
-  constexpr int kCW = kChunks == 1 ? 16 : 8, kPer = kChunks == 1 ? 1 : 4;
+  constexpr int kCW = VT::kCW, kPer = VT::kPer;
   const int G = p.G, N = p.n_rows, n_chunks = N / kCW;
   const uint32_t q_half_bytes = static_cast<uint32_t>(N) * 128u;  // between the two 64-column halves of Q
   FALCON_TRACE(tid == 0, 0);
@@ -394,7 +409,7 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
   // where it must: the softmax warps at once, because the loads everything waits for (Q, the
   // reference key, the tree) are theirs and their set-up can run under those loads; the producer
   // and the MMA warp after set-up that touches no global memory.
-  uint4 qreg[kChunks][2], kref[2];
+  uint4 qreg[VT::kQPasses][2], kref[2];
   int par_raw = -1;
   int n_early = 0;  // K/V tiles requested before the producer's wait
   if (warp >= kWarpSm0) {
@@ -405,8 +420,8 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
       // Q by plain loads (a TMA request would queue behind the K/V tiles already asked for), the
       // reference key (cache row 0) and the tree's parent array
 #pragma unroll
-      for (int pass = 0; pass < kChunks; ++pass) {
-        const int r = (st_id >> 3) + 64 * pass;
+      for (int pass = 0; pass < VT::kQPasses; ++pass) {
+        const int r = (st_id >> 3) + VT::kRowsPerPass * pass;
         qreg[pass][0] = qreg[pass][1] = make_uint4(0u, 0u, 0u, 0u);
         if (r < n_valid) {
           qreg[pass][0] = reinterpret_cast<const uint4*>(q_piece(r))[0];
@@ -601,8 +616,8 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
       // row: its scaled score against cache row 0 (8 threads per row, 16 columns each).
       const uint32_t kw[8] = {kref[0].x, kref[0].y, kref[0].z, kref[0].w, kref[1].x, kref[1].y, kref[1].z, kref[1].w};
 #pragma unroll
-      for (int pass = 0; pass < kChunks; ++pass) {
-        const int r = (st_id >> 3) + 64 * pass;
+      for (int pass = 0; pass < VT::kQPasses; ++pass) {
+        const int r = (st_id >> 3) + VT::kRowsPerPass * pass;
         if (r < N) {
           unsigned char* qrow = smem_gen + off_q + (q_part >> 2) * q_half_bytes + r * 128;
           const int u0 = 2 * (q_part & 3);
@@ -903,16 +918,16 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 
 bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
 
-template <int kChunks>
+template <int kVar>
 int pick_splits(falcon_ctx* ctx, int units, int max_tiles) {
-  int* resident = ctx->attn_resident[kChunks];
+  int* resident = ctx->attn_resident[1 + kVar];
   int best = 1;
   for (int s = kMaxSplits; s >= 1; --s) {
     if (s > max_tiles) continue;
     if (resident[s] == 0) {
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3(s, ctx->sm_count, 1);
-      cfg.blockDim = dim3(kThreads);
+      cfg.blockDim = dim3(Var<kVar>::kThreads);
       cfg.dynamicSmemBytes = kSmemMax;
       cudaLaunchAttribute attr;
       attr.id = cudaLaunchAttributeClusterDimension;
@@ -922,7 +937,7 @@ int pick_splits(falcon_ctx* ctx, int units, int max_tiles) {
       cfg.attrs = &attr;
       cfg.numAttrs = 1;
       int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, tree_attn_tck_kernel<kChunks, true>, &cfg) != cudaSuccess) n = -1;
+      if (cudaOccupancyMaxActiveClusters(&n, tree_attn_tck_kernel<kVar, true>, &cfg) != cudaSuccess) n = -1;
       resident[s] = n > 0 ? n : -1;
       cudaGetLastError();
     }
@@ -931,27 +946,27 @@ int pick_splits(falcon_ctx* ctx, int units, int max_tiles) {
   return best;
 }
 
-template <int kChunks>
+template <int kVar>
 int launch_impl(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s, int q_nodes) {
-  using C = Cfg<kChunks>;
+  using C = Cfg<Var<kVar>::kCfg>;
   const int B = a.tree.batch, Hq = a.n_q_heads, Hkv = a.n_kv_heads, G = Hq / Hkv;
   const int N = q_nodes * G;
   const int n_units = (a.tree.max_tree + q_nodes - 1) / q_nodes;
   if (static_cast<int64_t>(Hkv) * n_units > 65535) return FALCON_ERR_CAPACITY;
 
-  bool& attr_set = ctx->attn_attr_set[kChunks];
+  bool& attr_set = ctx->attn_attr_set[1 + kVar];
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(tree_attn_tck_kernel<kChunks, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(tree_attn_tck_kernel<kVar, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(kSmemMax));
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(tree_attn_tck_kernel<kChunks, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      e = cudaFuncSetAttribute(tree_attn_tck_kernel<kVar, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                static_cast<int>(kSmemMax));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaFuncSetAttribute(tree_attn_tck_kernel)");
     attr_set = true;
   }
   const int max_tiles = (a.tree.max_prefix_len + a.tree.max_tree + kBKMax - 1) / kBKMax;
   int splits = a.n_splits;
-  if (splits == 0) splits = pick_splits<kChunks>(ctx, Hkv * n_units * B, max_tiles > 0 ? max_tiles : 1);
+  if (splits == 0) splits = pick_splits<kVar>(ctx, Hkv * n_units * B, max_tiles > 0 ? max_tiles : 1);
   if (splits < 1) splits = 1;
   // Shared memory: Q, merge area (the other splits' shares of this CTA's head-dim rows and the row
   // sums) and the small arrays are fixed by the shape; the K/V ring takes the rest, as three stages
@@ -1036,7 +1051,7 @@ int launch_impl(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s, int 
 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(splits, Hkv * n_units, B);
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(Var<kVar>::kThreads);
   cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = s;
   cudaLaunchAttribute attr[2];
@@ -1049,8 +1064,8 @@ int launch_impl(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s, int 
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   cudaError_t e = (tile_keys == kBKMax && n_stages == 3)
-                      ? cudaLaunchKernelEx(&cfg, tree_attn_tck_kernel<kChunks, true>, mk, mv, mnk, mnv, p)
-                      : cudaLaunchKernelEx(&cfg, tree_attn_tck_kernel<kChunks, false>, mk, mv, mnk, mnv, p);
+                      ? cudaLaunchKernelEx(&cfg, tree_attn_tck_kernel<kVar, true>, mk, mv, mnk, mnv, p)
+                      : cudaLaunchKernelEx(&cfg, tree_attn_tck_kernel<kVar, false>, mk, mv, mnk, mnv, p);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tree_attn_tck_kernel launch");
   return FALCON_OK;
 }
@@ -1091,7 +1106,10 @@ bool tree_attn_tck_preferred(const falcon_ctx* ctx, const falcon_attn_args& a) {
 
 int launch_tree_attn_tck(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s) {
   const int G = a.n_q_heads / a.n_kv_heads, q_nodes = nodes_per_unit(a);
-  return q_nodes * G <= 64 ? launch_impl<1>(ctx, a, s, q_nodes) : launch_impl<2>(ctx, a, s, q_nodes);
+  const int rows = q_nodes * G;
+  if (rows <= 64) return launch_impl<0>(ctx, a, s, q_nodes);
+  if (rows <= 80) return launch_impl<1>(ctx, a, s, q_nodes);
+  return launch_impl<2>(ctx, a, s, q_nodes);
 }
 
 }  // namespace falcon
