@@ -95,6 +95,25 @@ def argmax(logits, vocab=None, n_threads=0):
     return g
 
 
+def lm_head_argmax(feat_bits, head_bits, hidden=None, want_logits=False, n_threads=0):
+    """feat_bits: uint16 (bf16 bit patterns) [N, feat_stride]; head_bits: uint16 [V, head_stride]; the first
+    `hidden` columns of both are used.  Returns (g [N] int32, best [N] float64[, logits [N, V] float64])."""
+    for a in (feat_bits, head_bits):
+        assert a.dtype == np.uint16 and a.ndim == 2 and a.flags.c_contiguous
+    N, fs = feat_bits.shape
+    V, hs = head_bits.shape
+    H = min(fs, hs) if hidden is None else hidden
+    g = np.empty(N, dtype=np.int32)
+    best = np.empty(N, dtype=np.float64)
+    logits = np.empty((N, V), dtype=np.float64) if want_logits else None
+    rc = lib().oracle_lm_head_argmax(_p(feat_bits, C.c_uint16), C.c_int64(fs), _p(head_bits, C.c_uint16), C.c_int64(hs),
+                                     C.c_int32(N), C.c_int32(H), C.c_int32(V), _p(g, C.c_int32), _p(best, C.c_double),
+                                     _p(logits, C.c_double) if want_logits else None, C.c_int(n_threads))
+    if rc:
+        raise ValueError("oracle_lm_head_argmax failed: %d" % rc)
+    return (g, best, logits) if want_logits else (g, best)
+
+
 def topm(logits, m, vocab=None, n_threads=0):
     """logits: C-contiguous fp32 [N, stride].  Returns (values [N, m] fp32, indices [N, m] int32), best first."""
     assert logits.dtype == np.float32 and logits.ndim == 2 and logits.flags.c_contiguous

@@ -254,6 +254,44 @@ int oracle_argmax(const float* logits, int32_t N, int32_t V, int64_t stride, int
   return 0;
 }
 
+// LM-head logits of the tree's nodes and their greedy argmax without a logits matrix in
+// between.  The verification pass ends in the target model's LM head: "the LM Head computes
+// the probability distribution based on the aggregated features" (Section 3.1) and Eq. 6 writes
+// p = Softmax(LM(f)); with temperature 0 (Section 4.1) only the position of the largest logit
+// is needed, and the softmax does not move it.  The LM head is taken as a bias-free linear map
+// (the LLaMA / Vicuna heads the paper evaluates have no bias):
+//   logit[i, v] = sum_k feat[i, k] * head[v, k],      g[i] = lowest v attaining max_v logit[i, v].
+// feat: bf16 bit patterns [N, feat_stride], head: bf16 [V, head_stride] (both row-major, the
+// first `hidden` columns used).  Products of bf16 values are exact in double and the sum runs
+// over k in order in double.  Same tie and NaN rules as oracle_argmax (strict '>' scan).
+// best[i] (optional) receives the winning logit; logits_out (optional, [N, V] doubles) all of them.
+int oracle_lm_head_argmax(const uint16_t* feat, int64_t feat_stride, const uint16_t* head, int64_t head_stride, int32_t N,
+                          int32_t hidden, int32_t V, int32_t* g, double* best, double* logits_out, int n_threads) {
+  if (N < 0 || hidden < 1 || V < 1 || feat_stride < hidden || head_stride < hidden) return 1;
+  const int nt = pick_threads(n_threads);
+  (void)nt;
+#pragma omp parallel for num_threads(nt)
+  for (int32_t i = 0; i < N; ++i) {
+    const uint16_t* f = feat + static_cast<int64_t>(i) * feat_stride;
+    double top = -std::numeric_limits<double>::infinity();
+    int32_t idx = 0;
+    for (int32_t v = 0; v < V; ++v) {
+      const uint16_t* w = head + static_cast<int64_t>(v) * head_stride;
+      double acc = 0.0;
+      for (int32_t k = 0; k < hidden; ++k)
+        acc += static_cast<double>(bf16_to_float(f[k])) * static_cast<double>(bf16_to_float(w[k]));
+      if (logits_out) logits_out[static_cast<int64_t>(i) * V + v] = acc;
+      if (acc > top) {
+        top = acc;
+        idx = v;
+      }
+    }
+    g[i] = idx;
+    if (best) best[i] = top;
+  }
+  return 0;
+}
+
 // Top-m entries of every row, best first: the children a tree node is given when the tree is
 // grown ("the m tokens with the highest probability", Appendix A; m = 20 at the root there).
 // Plain definition: m passes over the row, each taking the best entry not taken yet.  Order:

@@ -623,3 +623,89 @@ def test_feature_gather_rejects_bad_paths():
         oracle.feature_gather([0, 4], path, [2], [1, 2, 3, 4], feat)
     with pytest.raises(ValueError):
         oracle.feature_gather([0, 4], np.array([[0, 1, 2, 3]], np.int32), [5], [1, 2, 3, 4], feat)
+
+
+# --------------------------------------------------------------------------- LM-head argmax (Section 3.1, Eq. 6)
+def _bits(x):
+    return synth.f32_to_bf16_bits(np.asarray(x, dtype=np.float32))
+
+
+def test_lm_head_argmax_hand_worked():
+    c = GOLD["lm_head_argmax_basic"]
+    g, best, logits = oracle.lm_head_argmax(_bits(c["features"]), _bits(c["head"]), want_logits=True)
+    assert np.array_equal(logits, np.array(c["expected_logits"], dtype=np.float64))
+    assert g.tolist() == c["expected_argmax"]          # node 0: three-way tie, the lowest index wins
+    assert best.tolist() == c["expected_best"]
+
+
+def test_lm_head_logits_are_the_matrix_product_with_the_head_transposed():
+    rng = np.random.default_rng(3)
+    N, H, V = 7, 96, 53                                 # all different: a transposed operand cannot pass
+    f = synth.normal_bf16(rng, (N, H))
+    w = synth.normal_bf16(rng, (V, H))
+    g, best, logits = oracle.lm_head_argmax(f, w, want_logits=True)
+    ref = synth.bf16_bits_to_f32(f).astype(np.float64) @ synth.bf16_bits_to_f32(w).astype(np.float64).T
+    assert np.allclose(logits, ref, rtol=1e-12, atol=1e-12)
+    assert np.array_equal(g, np.argmax(ref, axis=1))
+    assert np.array_equal(best, logits[np.arange(N), g])
+
+
+def test_lm_head_integer_data_is_exact_and_ties_go_to_the_lowest_index():
+    rng = np.random.default_rng(4)
+    N, H, V = 9, 64, 40
+    fi = rng.integers(-3, 4, size=(N, H))
+    wi = rng.integers(-3, 4, size=(V, H))
+    wi[17] = wi[5]                                      # two identical head rows: equal logits for every node
+    g, best, logits = oracle.lm_head_argmax(_bits(fi), _bits(wi), want_logits=True)
+    ref = fi.astype(np.int64) @ wi.astype(np.int64).T
+    assert np.array_equal(logits, ref.astype(np.float64))
+    assert np.array_equal(g, np.argmax(ref, axis=1))    # numpy also returns the first maximum
+    assert not np.any(g == 17)
+
+
+def test_lm_head_one_hot_feature_reads_back_a_head_column():
+    rng = np.random.default_rng(5)
+    H, V = 32, 77
+    w = synth.normal_bf16(rng, (V, H))
+    f = np.zeros((H, H), dtype=np.float32)
+    f[np.arange(H), np.arange(H)] = 1.0                 # node k = unit vector e_k -> logits = head[:, k]
+    g, best, logits = oracle.lm_head_argmax(_bits(f), w, want_logits=True)
+    col = synth.bf16_bits_to_f32(w).astype(np.float64)
+    assert np.array_equal(logits, col.T)
+    assert np.array_equal(g, np.argmax(col, axis=0))
+
+
+def test_lm_head_row_strides_nan_and_signed_zero():
+    rng = np.random.default_rng(6)
+    N, H, V = 5, 24, 31
+    f = synth.normal_bf16(rng, (N, H + 8))              # junk beyond `hidden` must not be read
+    w = synth.normal_bf16(rng, (V, H + 16))
+    g, best = oracle.lm_head_argmax(f, w, hidden=H)
+    g2, best2 = oracle.lm_head_argmax(np.ascontiguousarray(f[:, :H]), np.ascontiguousarray(w[:, :H]))
+    assert np.array_equal(g, g2) and np.array_equal(best, best2)
+    # a head row holding a NaN gives NaN logits, which never win; all rows NaN -> index 0
+    wn = np.ascontiguousarray(w[:, :H]).copy()
+    wn[int(g2[0]), 3] = 0x7FC0
+    g3, _ = oracle.lm_head_argmax(np.ascontiguousarray(f[:, :H]), wn)
+    assert g3[0] != g2[0]
+    wn[:, 3] = 0x7FC0
+    g4, _ = oracle.lm_head_argmax(np.ascontiguousarray(f[:, :H]), wn)
+    assert np.all(g4 == 0)
+    # -0 and +0 logits tie: features of zeros against any head -> every logit is a zero -> index 0
+    z = np.zeros((2, H), dtype=np.uint16)
+    z[1, :] = 0x8000
+    g5, best5 = oracle.lm_head_argmax(z, np.ascontiguousarray(w[:, :H]))
+    assert np.all(g5 == 0) and np.all(best5 == 0.0)
+
+
+def test_lm_head_argmax_agrees_with_the_logits_scan():
+    # the fused definition and "materialise fp32 logits, then oracle.argmax" pick the same token when the margin
+    # between the two best logits is far above fp32 rounding
+    rng = np.random.default_rng(7)
+    N, H, V = 12, 128, 300
+    f = synth.normal_bf16(rng, (N, H))
+    w = synth.normal_bf16(rng, (V, H))
+    g, best, logits = oracle.lm_head_argmax(f, w, want_logits=True)
+    srt = np.sort(logits, axis=1)
+    assert np.all(srt[:, -1] - srt[:, -2] > 1e-3)
+    assert np.array_equal(g, oracle.argmax(np.ascontiguousarray(logits.astype(np.float32))))
