@@ -189,8 +189,10 @@ typedef struct {
   falcon_tree_desc tree;
   int32_t vocab;
   int64_t logits_stride;  /* elements between rows, >= vocab                          */
-  const float* logits;    /* fp32 [N, logits_stride]                                  */
-  int32_t* argmax_out;    /* [N] g, always written                                    */
+  const float* logits;    /* fp32 [N, logits_stride]; NULL: g is given, see argmax_out */
+  int32_t* argmax_out;    /* [N] g: written; with logits == NULL it is read instead   */
+                          /* (e.g. what falcon_lm_head_argmax left there), vocab and  */
+                          /* logits_stride are ignored and only the search runs       */
   int32_t* path;          /* [B, path_stride]                                         */
   int32_t path_stride;    /* >= max_tree                                              */
   int32_t* n_path;        /* [B]                                                      */
@@ -198,6 +200,44 @@ typedef struct {
 } falcon_accept_args;
 
 int falcon_tree_accept(falcon_ctx* ctx, const falcon_accept_args* args, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * falcon_lm_head_argmax - the greedy token of every tree node straight from the
+ * LM head (Section 3.1: "the LM Head computes the probability distribution based
+ * on the aggregated features"; Eq. 6: p = Softmax(LM(f)); at temperature 0,
+ * Section 4.1, only the position of the largest logit matters).  The [N, vocab]
+ * logits are never written to memory:
+ *
+ *   logit[i, v]   = sum_k features[i, k] * lm_head[v, k]     (bf16 inputs, fp32 sums)
+ *   argmax_out[i] = lowest v attaining the maximum (NaN never wins; a row with
+ *                   nothing above -inf gives 0)
+ *   max_out[i]    = that logit (optional)
+ *
+ * The head is a bias-free linear map stored row by row ([vocab, hidden], what the
+ * LLaMA / Vicuna checkpoints hold).  falcon_tree_accept with logits == NULL then
+ * finds the accepted path from argmax_out.  The sums are taken in fp32 in the
+ * tensor core's order: two logits closer than that rounding may swap places
+ * relative to an exact evaluation.
+ *   limits   n_rows <= 65535; both pitches multiples of 8 elements and both bases
+ *            16-byte aligned (FALCON_ERR_UNSUPPORTED otherwise)
+ *   status   optional device word; FALCON_DEV_TIMEOUT is set there if a bounded
+ *            wait inside the kernel gave up (the results are then not valid)
+ * Device pointers; the caller owns every buffer; scratch comes from the context.
+ * ------------------------------------------------------------------------- */
+typedef struct {
+  int32_t n_rows;         /* N: rows of `features` (tree nodes)                        */
+  int32_t hidden;
+  int32_t vocab;
+  const void* features;   /* bf16 [n_rows, feat_stride]                                */
+  int64_t feat_stride;    /* elements between rows, >= hidden                          */
+  const void* lm_head;    /* bf16 [vocab, head_stride]                                 */
+  int64_t head_stride;    /* elements between rows, >= hidden                          */
+  int32_t* argmax_out;    /* [n_rows]                                                  */
+  float* max_out;         /* [n_rows] or NULL                                          */
+  int32_t* status;        /* 1 word or NULL                                            */
+} falcon_lm_argmax_args;
+
+int falcon_lm_head_argmax(falcon_ctx* ctx, const falcon_lm_argmax_args* args, void* stream);
 
 /* ---------------------------------------------------------------------------
  * falcon_topm - the m best entries of every logits row, best first: the children

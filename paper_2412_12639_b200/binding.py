@@ -56,6 +56,12 @@ class TopmArgs(C.Structure):
                 ("m", C.c_int32), ("top_val", C.c_void_p), ("top_idx", C.c_void_p)]
 
 
+class LmArgmaxArgs(C.Structure):
+    _fields_ = [("n_rows", C.c_int32), ("hidden", C.c_int32), ("vocab", C.c_int32), ("features", C.c_void_p),
+                ("feat_stride", C.c_int64), ("lm_head", C.c_void_p), ("head_stride", C.c_int64),
+                ("argmax_out", C.c_void_p), ("max_out", C.c_void_p), ("status", C.c_void_p)]
+
+
 class GatherArgs(C.Structure):
     _fields_ = [("tree", TreeDesc), ("hidden", C.c_int32), ("feat_stride", C.c_int64), ("features", C.c_void_p),
                 ("path", C.c_void_p), ("path_stride", C.c_int32), ("n_path", C.c_void_p), ("out_rows", C.c_int32),
@@ -95,7 +101,7 @@ def load_library():
     lib.falcon_tree_validate_host.restype = C.c_int
     for name, argt in (("falcon_tree_attn", AttnArgs), ("falcon_tree_accept", AcceptArgs),
                        ("falcon_kv_compact", CompactArgs), ("falcon_topm", TopmArgs),
-                       ("falcon_feature_gather", GatherArgs)):
+                       ("falcon_feature_gather", GatherArgs), ("falcon_lm_head_argmax", LmArgmaxArgs)):
         fn = getattr(lib, name)
         fn.argtypes = [C.c_void_p, C.POINTER(argt), C.c_void_p]
         fn.restype = C.c_int
@@ -207,6 +213,12 @@ class Context:
             self._check(rc, "falcon_topm")
         return rc
 
+    def falcon_lm_head_argmax(self, args: LmArgmaxArgs, stream=None, check: bool = True) -> int:
+        rc = self._lib.falcon_lm_head_argmax(self._h, C.byref(args), _stream(stream))
+        if check:
+            self._check(rc, "falcon_lm_head_argmax")
+        return rc
+
     def falcon_feature_gather(self, args: GatherArgs, stream=None, check: bool = True) -> int:
         rc = self._lib.falcon_feature_gather(self._h, C.byref(args), _stream(stream))
         if check:
@@ -238,6 +250,12 @@ def accept_args(tree: TreeDesc, vocab, logits, logits_stride, argmax_out, path, 
 
 def topm_args(n_rows, vocab, logits, logits_stride, m, top_val, top_idx) -> TopmArgs:
     return TopmArgs(n_rows, vocab, logits_stride, _ptr(logits), m, _ptr(top_val), _ptr(top_idx))
+
+
+def lm_argmax_args(n_rows, hidden, vocab, features, feat_stride, lm_head, head_stride, argmax_out, max_out=None,
+                   status=None) -> LmArgmaxArgs:
+    return LmArgmaxArgs(n_rows, hidden, vocab, _ptr(features), feat_stride, _ptr(lm_head), head_stride,
+                        _ptr(argmax_out), _ptr(max_out), _ptr(status))
 
 
 def gather_args(tree: TreeDesc, hidden, features, feat_stride, path, path_stride, n_path, out_rows, features_out,

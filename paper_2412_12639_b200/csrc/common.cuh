@@ -32,6 +32,7 @@ struct falcon_ctx {
   // (0 = not asked yet, -1 = none).  Index 0: rows-on-lanes kernel; 1-3: the keys-on-lanes kernel's
   // three variants.
   bool attn_attr_set[4] = {false, false, false, false};
+  bool lm_attr_set = false;  // the same for the LM-head kernel
   int attn_resident[4][9] = {};
 };
 
@@ -48,6 +49,8 @@ int launch_kv_compact(falcon_ctx* ctx, const falcon_compact_args& a, cudaStream_
 int launch_feature_gather(falcon_ctx* ctx, const falcon_gather_args& a, cudaStream_t s);
 int check_gather_args(const falcon_gather_args& g, int max_tree);
 int launch_tree_topm(falcon_ctx* ctx, const falcon_topm_args& a, cudaStream_t s);
+int launch_tree_search(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_t s);
+int launch_lm_head_argmax(falcon_ctx* ctx, const falcon_lm_argmax_args& a, cudaStream_t s);
 int launch_tree_attn_simt(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s);
 int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s);
 bool tree_attn_tc_supports(const falcon_ctx* ctx, const falcon_attn_args& a);

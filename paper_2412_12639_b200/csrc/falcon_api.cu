@@ -189,11 +189,24 @@ int falcon_tree_accept(falcon_ctx* ctx, const falcon_accept_args* a, void* strea
   if (!ctx || !a) return FALCON_ERR_INVALID_ARG;
   int rc = check_tree_desc(a->tree, true);
   if (rc) return rc;
-  if (!a->logits || !a->argmax_out || !a->path || !a->n_path || !a->next_token) return FALCON_ERR_INVALID_ARG;
-  if (a->vocab < 1 || a->logits_stride < a->vocab) return FALCON_ERR_INVALID_ARG;
+  if (!a->argmax_out || !a->path || !a->n_path || !a->next_token) return FALCON_ERR_INVALID_ARG;
   if (a->path_stride < a->tree.max_tree) return FALCON_ERR_INVALID_ARG;
+  if (!a->logits) return launch_tree_search(ctx, *a, static_cast<cudaStream_t>(stream));  // g is given
+  if (a->vocab < 1 || a->logits_stride < a->vocab) return FALCON_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(a->logits) & 3) return FALCON_ERR_INVALID_ARG;
   return launch_tree_accept(ctx, *a, static_cast<cudaStream_t>(stream));
+}
+
+int falcon_lm_head_argmax(falcon_ctx* ctx, const falcon_lm_argmax_args* a, void* stream) {
+  if (!ctx || !a) return FALCON_ERR_INVALID_ARG;
+  if (!a->features || !a->lm_head || !a->argmax_out) return FALCON_ERR_INVALID_ARG;
+  if (a->n_rows < 1 || a->hidden < 1 || a->vocab < 1) return FALCON_ERR_INVALID_ARG;
+  if (a->feat_stride < a->hidden || a->head_stride < a->hidden) return FALCON_ERR_INVALID_ARG;
+  // TMA: 16-byte aligned bases and row pitches
+  if ((a->feat_stride | a->head_stride) & 7) return FALCON_ERR_UNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(a->features) | reinterpret_cast<uintptr_t>(a->lm_head)) & 15) return FALCON_ERR_UNSUPPORTED;
+  if (a->n_rows > 65535) return FALCON_ERR_CAPACITY;
+  return launch_lm_head_argmax(ctx, *a, static_cast<cudaStream_t>(stream));
 }
 
 int falcon_topm(falcon_ctx* ctx, const falcon_topm_args* a, void* stream) {

@@ -48,6 +48,61 @@ __device__ __forceinline__ void take(Best& s, float x, int i) {
   }
 }
 
+// The longest accepted path of sequence b from the nodes' argmax tokens: thread tid < T brings
+// g = the argmax of node tid; every thread of the CTA calls this.
+__device__ __forceinline__ void search_tree(const AcceptParams& p, int b, int base, int T_real, int g, int* s_par, int* s_tok,
+                                            int* s_g, int* s_key) {
+  const int tid = threadIdx.x;
+  const int T = min(T_real, FALCON_T_MAX);
+  bool bad = (T_real > FALCON_T_MAX);
+  if (tid < T) {
+    s_g[tid] = g;
+    const int pr = p.parent[base + tid];
+    s_par[tid] = pr;
+    s_tok[tid] = p.token[base + tid];
+    bad = bad || ((tid == 0) ? (pr != -1) : (pr < 0 || pr >= tid));
+  }
+  const int any_bad = __syncthreads_or(bad ? 1 : 0);
+
+  // alive(c): every non-root node on the chain root..c carries the argmax of its parent
+  int key = -1;
+  if (tid < T && !any_bad) {
+    bool alive = true;
+    int depth = 0, u = tid;
+    while (u != 0 && depth < T) {
+      const int pu = s_par[u];
+      alive = alive && (s_tok[u] == s_g[pu]);
+      u = pu;
+      ++depth;
+    }
+    if (alive) key = depth * 256 + (255 - tid);  // deeper wins, then the lower index
+  }
+  if (tid == 0 && any_bad) key = 255;  // malformed tree: root only
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xffffffffu, key, o));
+  if ((tid & 31) == 0) s_key[tid >> 5] = key;
+  __syncthreads();
+  key = s_key[0];
+#pragma unroll
+  for (int w = 1; w < kAcceptThreads / 32; ++w) key = max(key, s_key[w]);
+  const int best = 255 - (key & 255);
+  const int n = (key >> 8) + 1;
+
+  int32_t* prow = p.path + static_cast<int64_t>(b) * p.path_stride;
+  for (int j = n + tid; j < p.path_stride; j += kAcceptThreads) prow[j] = -1;
+  if (tid == 0) {
+    int u = best;
+    for (int j = n - 1; j >= 0; --j) {
+      prow[j] = u;
+      u = s_par[u];
+    }
+    p.n_path[b] = n;
+    p.next_token[b] = s_g[best];
+    if (any_bad) dev_status_or(p.status, b, FALCON_DEV_BAD_TREE);
+  }
+}
+
+
 __global__ void __launch_bounds__(kAcceptThreads) tree_accept_kernel(const AcceptParams p) {
   __shared__ Best warp_best[kAcceptThreads / 32];
   __shared__ int s_flag;
@@ -117,7 +172,7 @@ __global__ void __launch_bounds__(kAcceptThreads) tree_accept_kernel(const Accep
   __threadfence();
 
   // ---- last CTA of sequence b: fold the partials, then search the tree ----
-  bool bad = (T_real > FALCON_T_MAX);
+  int g = 0;
   if (tid < T) {
     Best r{-INFINITY, kNone};
     const int64_t o = static_cast<int64_t>(base + tid) * p.chunks;
@@ -133,53 +188,24 @@ __global__ void __launch_bounds__(kAcceptThreads) tree_accept_kernel(const Accep
 #pragma unroll
       for (int k = 0; k < 8; ++k) r = merge(r, Best{v[k], ix[k]});
     }
-    const int g = (r.i == kNone) ? 0 : r.i;
+    g = (r.i == kNone) ? 0 : r.i;
     p.argmax_out[base + tid] = g;
-    s_g[tid] = g;
-    const int pr = p.parent[base + tid];
-    s_par[tid] = pr;
-    s_tok[tid] = p.token[base + tid];
-    bad = bad || ((tid == 0) ? (pr != -1) : (pr < 0 || pr >= tid));
   }
-  const int any_bad = __syncthreads_or(bad ? 1 : 0);
+  search_tree(p, b, base, T_real, g, s_par, s_tok, s_g, s_key);
+  if (tid == 0) p.tickets[b] = 0;  // ready for the next call
+}
 
-  // alive(c): every non-root node on the chain root..c carries the argmax of its parent
-  int key = -1;
-  if (tid < T && !any_bad) {
-    bool alive = true;
-    int depth = 0, u = tid;
-    while (u != 0 && depth < T) {
-      const int pu = s_par[u];
-      alive = alive && (s_tok[u] == s_g[pu]);
-      u = pu;
-      ++depth;
-    }
-    if (alive) key = depth * 256 + (255 - tid);  // deeper wins, then the lower index
-  }
-  if (tid == 0 && any_bad) key = 255;  // malformed tree: root only
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xffffffffu, key, o));
-  if ((tid & 31) == 0) s_key[tid >> 5] = key;
-  __syncthreads();
-  key = s_key[0];
-#pragma unroll
-  for (int w = 1; w < kAcceptThreads / 32; ++w) key = max(key, s_key[w]);
-  const int best = 255 - (key & 255);
-  const int n = (key >> 8) + 1;
-
-  int32_t* prow = p.path + static_cast<int64_t>(b) * p.path_stride;
-  for (int j = n + tid; j < p.path_stride; j += kAcceptThreads) prow[j] = -1;
-  if (tid == 0) {
-    int u = best;
-    for (int j = n - 1; j >= 0; --j) {
-      prow[j] = u;
-      u = s_par[u];
-    }
-    p.n_path[b] = n;
-    p.next_token[b] = s_g[best];
-    if (any_bad) dev_status_or(p.status, b, FALCON_DEV_BAD_TREE);
-    p.tickets[b] = 0;  // ready for the next call
-  }
+// The search alone, for callers that already have g (falcon_lm_head_argmax writes it): one CTA per
+// sequence.
+__global__ void __launch_bounds__(kAcceptThreads) tree_search_kernel(const AcceptParams p) {
+  __shared__ int s_par[FALCON_T_MAX], s_tok[FALCON_T_MAX], s_g[FALCON_T_MAX];
+  __shared__ int s_key[kAcceptThreads / 32];
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const int base = p.node_off[b];
+  const int T_real = p.node_off[b + 1] - base;
+  const int g = tid < min(T_real, FALCON_T_MAX) ? p.argmax_out[base + tid] : 0;
+  search_tree(p, b, base, T_real, g, s_par, s_tok, s_g, s_key);
 }
 
 constexpr int kAcceptMaxChunks = 64;  // vocabulary chunks per row at most (the static scratch is sized by it)
@@ -250,6 +276,24 @@ int launch_tree_accept(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_
   cfg.numAttrs = 1;
   cudaError_t e = cudaLaunchKernelEx(&cfg, tree_accept_kernel, p);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tree_accept_kernel launch");
+  return FALCON_OK;
+}
+
+// The nodes' argmax tokens are already in a.argmax_out (written by an earlier call on the stream):
+// the path search alone, one CTA per sequence.
+int launch_tree_search(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_t s) {
+  const AcceptParams p = accept_params(a, 1, 4, nullptr, nullptr);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(a.tree.batch);
+  cfg.blockDim = dim3(kAcceptThreads);
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, tree_search_kernel, p);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "tree_search_kernel launch");
   return FALCON_OK;
 }
 

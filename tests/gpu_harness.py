@@ -168,3 +168,18 @@ def run_compact(dt: DevTrees, Hkv, D, k_layers, v_layers, path, n_path, k_tree_l
     ctx().falcon_kv_compact(a)
     torch.cuda.synchronize()
     return [host_bits(t) for t in kd], [host_bits(t) for t in vd], new_len.cpu().numpy()
+
+
+def run_lm_argmax(feat_bits, head_bits, hidden=None, check=True):
+    """falcon_lm_head_argmax on uint16 bf16 bit patterns [N, feat_stride] / [V, head_stride].
+    Returns (argmax [N], max [N] fp32, status word, rc)."""
+    N, fs = feat_bits.shape
+    V, hs = head_bits.shape
+    Hd = min(fs, hs) if hidden is None else hidden
+    f, w = dev_bf16(feat_bits), dev_bf16(head_bits)
+    g = torch.full((N,), -3, dtype=torch.int32, device="cuda")
+    mx = torch.full((N,), -7.0, dtype=torch.float32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rc = ctx().falcon_lm_head_argmax(binding.lm_argmax_args(N, Hd, V, f, fs, w, hs, g, mx, st), check=check)
+    torch.cuda.synchronize()
+    return g.cpu().numpy(), mx.cpu().numpy(), int(st.item()), rc

@@ -54,7 +54,8 @@ def test_binding_structs_match_header_field_order():
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     for cname, struct in (("falcon_tree_desc", binding.TreeDesc), ("falcon_attn_args", binding.AttnArgs),
                           ("falcon_accept_args", binding.AcceptArgs), ("falcon_compact_args", binding.CompactArgs),
-                          ("falcon_gather_args", binding.GatherArgs)):
+                          ("falcon_gather_args", binding.GatherArgs),
+                          ("falcon_lm_argmax_args", binding.LmArgmaxArgs)):
         end = re.search(r"\}\s*%s;" % cname, text).start()
         body = text[text.rfind("typedef struct {", 0, end) + len("typedef struct {"):end]
         fields = []
@@ -78,7 +79,8 @@ def test_binding_structs_match_the_compiled_layout(tmp_path):
         pytest.skip("no C compiler")
     structs = (("falcon_tree_desc", binding.TreeDesc), ("falcon_attn_args", binding.AttnArgs),
                ("falcon_accept_args", binding.AcceptArgs), ("falcon_topm_args", binding.TopmArgs),
-               ("falcon_compact_args", binding.CompactArgs), ("falcon_gather_args", binding.GatherArgs))
+               ("falcon_compact_args", binding.CompactArgs), ("falcon_gather_args", binding.GatherArgs),
+               ("falcon_lm_argmax_args", binding.LmArgmaxArgs))
     lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "falcon.h"', 'int main(void) {']
     for cname, st in structs:
         lines.append('  printf("%s %%zu\\n", sizeof(%s));' % (cname, cname))

@@ -636,6 +636,124 @@ def test_topm_rejects_bad_arguments_without_launching():
     assert (idx.cpu().numpy() == -7).all() and (val.cpu().numpy() == 3.0).all()
 
 
+# ------------------------------------------------------------------------ LM-head argmax (Section 3.1, Eq. 6)
+def assert_lm_argmax(f, w, hidden=None, tol=None):
+    """The kernel sums in fp32 in the tensor core's order, the oracle in double: the maximum itself must agree
+    within the rounding of those sums, and where the two pick different tokens the oracle's logit of the
+    kernel's token must lie within that rounding of the oracle's maximum (both are then valid greedy tokens)."""
+    g_ref, best_ref, logits = oracle.lm_head_argmax(f, w, hidden=hidden, want_logits=True)
+    g, mx, status, rc = H.run_lm_argmax(f, w, hidden=hidden)
+    assert rc == 0 and status == 0
+    Hd = min(f.shape[1], w.shape[1]) if hidden is None else hidden
+    if tol is None:
+        # |sum error| <= hidden * 2^-24 * sum |a b| (fp32 accumulation of exact products), with slack 4
+        fa = np.abs(synth.bf16_bits_to_f32(f[:, :Hd]).astype(np.float64))
+        wa = np.abs(synth.bf16_bits_to_f32(w[:, :Hd]).astype(np.float64))
+        tol = 4.0 * Hd * 2.0 ** -24 * float((fa.max(axis=0) * wa.max(axis=0)).sum())
+    assert g.min() >= 0 and g.max() < w.shape[0]
+    at_gpu = logits[np.arange(len(g)), g]
+    assert np.all(best_ref - at_gpu <= tol), (np.max(best_ref - at_gpu), tol)
+    assert np.all(np.abs(mx.astype(np.float64) - at_gpu) <= tol)
+    return g, g_ref
+
+
+@pytest.mark.parametrize("N,Hd,V", [(60, 256, 1000), (7, 64, 40), (130, 192, 3001), (300, 128, 2500), (60, 128, 50000)])
+def test_lm_head_argmax_integer_data_is_bit_exact(N, Hd, V):
+    # small integers: every product and every partial sum is exact in fp32, so values, ties and indices must
+    # equal the oracle's bit for bit (one node tile, two resident tiles, three tiles in two rounds; a vocabulary
+    # run longer than one MMA tile per CTA; vocabulary and node tails)
+    rng = np.random.default_rng(N + V)
+    fi = rng.integers(-3, 4, size=(N, Hd))
+    wi = rng.integers(-3, 4, size=(V, Hd))
+    wi[V // 2] = wi[5]                                         # identical head rows: a tie for every node
+    wi[V - 1] = wi[5]
+    f = synth.f32_to_bf16_bits(fi.astype(np.float32))
+    w = synth.f32_to_bf16_bits(wi.astype(np.float32))
+    g_ref, best_ref = oracle.lm_head_argmax(f, w)
+    for _ in range(2):                                         # twice: the arrival counter must come back to zero
+        g, mx, status, rc = H.run_lm_argmax(f, w)
+        assert rc == 0 and status == 0
+        np.testing.assert_array_equal(g, g_ref)
+        np.testing.assert_array_equal(mx.astype(np.float64), best_ref)
+
+
+@pytest.mark.parametrize("N,Hd,V,pad", [(60, 512, 5000, 0), (130, 320, 3001, 8), (15, 72, 1000, 24), (257, 256, 4096, 0)])
+def test_lm_head_argmax_random_data(N, Hd, V, pad):
+    # hidden sizes that are not multiples of the 64-column stage, padded row pitches, ragged tails
+    rng = np.random.default_rng(N * 7 + V)
+    f = synth.normal_bf16(rng, (N, Hd + pad))
+    w = synth.normal_bf16(rng, (V, Hd + pad))
+    g, g_ref = assert_lm_argmax(f, w, hidden=Hd)
+    assert np.mean(g == g_ref) > 0.95                          # near-ties are rare with continuous data
+
+
+def test_lm_head_argmax_special_values():
+    rng = np.random.default_rng(11)
+    N, Hd, V = 20, 128, 700
+    f = synth.normal_bf16(rng, (N, Hd))
+    w = synth.normal_bf16(rng, (V, Hd))
+    g0, _ = oracle.lm_head_argmax(f, w)
+    wn = w.copy()
+    wn[int(g0[0]), 3] = 0x7FC0                                 # the winner's head row gets a NaN: it cannot win
+    g_ref, best_ref = oracle.lm_head_argmax(f, wn)
+    g, mx, status, rc = H.run_lm_argmax(f, wn)
+    assert rc == 0 and status == 0 and g[0] != g0[0]
+    np.testing.assert_array_equal(g, g_ref)
+    wn[:, 3] = 0x7FC0                                          # every logit NaN: index 0
+    g, mx, status, rc = H.run_lm_argmax(f, wn)
+    assert np.all(g == 0)
+    z = np.zeros((4, Hd), dtype=np.uint16)                     # zero features: every logit is a zero, index 0
+    z[1] = 0x8000
+    g, mx, status, rc = H.run_lm_argmax(z, w)
+    assert np.all(g == 0) and np.all(mx == 0.0)
+
+
+def test_lm_head_argmax_then_accept_from_the_argmax():
+    # verification without a logits matrix: the LM-head call writes g, the acceptance call with logits == NULL
+    # searches the tree with it
+    rng = np.random.default_rng(21)
+    tb = H.make_trees([20, 33, 7], [5, 9, 0], rng, vocab=50)
+    N, Hd, V = tb.total_nodes, 128, 50
+    fi = rng.integers(-3, 4, size=(N, Hd))
+    wi = rng.integers(-3, 4, size=(V, Hd))
+    f = synth.f32_to_bf16_bits(fi.astype(np.float32))
+    w = synth.f32_to_bf16_bits(wi.astype(np.float32))
+    g_ref, _ = oracle.lm_head_argmax(f, w)
+    for b in range(tb.batch):                                  # plant matches: a child carries its parent's argmax
+        o = int(tb.node_off[b])
+        for i in range(1, int(tb.node_off[b + 1]) - o):
+            if rng.random() < 0.6:
+                tb.token[o + i] = g_ref[o + tb.parent[o + i]]
+    dt = H.DevTrees(tb)
+    fd, wd = H.dev_bf16(f), H.dev_bf16(w)
+    g = torch.zeros(N, dtype=torch.int32, device="cuda")
+    path = torch.full((tb.batch, 64), -9, dtype=torch.int32, device="cuda")
+    n_path = torch.zeros(tb.batch, dtype=torch.int32, device="cuda")
+    nxt = torch.zeros(tb.batch, dtype=torch.int32, device="cuda")
+    c = H.ctx()
+    c.falcon_lm_head_argmax(binding.lm_argmax_args(N, Hd, V, fd, Hd, wd, Hd, g))
+    c.falcon_tree_accept(binding.accept_args(dt.desc(), 0, None, 0, g, path, 64, n_path, nxt))
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(g.cpu().numpy(), g_ref)
+    rp, rn, rt = oracle.tree_accept(tb.node_off, tb.parent, tb.token, g_ref, path_stride=64)
+    np.testing.assert_array_equal(path.cpu().numpy(), rp)
+    np.testing.assert_array_equal(n_path.cpu().numpy(), rn)
+    np.testing.assert_array_equal(nxt.cpu().numpy(), rt)
+
+
+def test_lm_head_argmax_rejects_bad_arguments_without_launching():
+    f = torch.zeros((4, 72), dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros((10, 72), dtype=torch.bfloat16, device="cuda")
+    g = torch.full((4,), -5, dtype=torch.int32, device="cuda")
+    c = H.ctx()
+    assert c.falcon_lm_head_argmax(binding.lm_argmax_args(4, 72, 10, f, 64, w, 72, g), check=False) == binding.ERR_INVALID_ARG
+    assert c.falcon_lm_head_argmax(binding.lm_argmax_args(4, 70, 10, f, 70, w, 72, g), check=False) == binding.ERR_UNSUPPORTED
+    assert c.falcon_lm_head_argmax(binding.lm_argmax_args(0, 72, 10, f, 72, w, 72, g), check=False) == binding.ERR_INVALID_ARG
+    assert c.falcon_lm_head_argmax(binding.lm_argmax_args(4, 72, 10, f, 72, w, 72, None), check=False) == binding.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert (g.cpu().numpy() == -5).all()
+
+
 # ------------------------------------------------------------------------ ABI
 def test_abi_rejects_bad_arguments_without_launching():
     rng = np.random.default_rng(1)
