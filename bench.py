@@ -254,6 +254,43 @@ def time_topm(ctx, binding, torch, dev, stream, logits_h, peak, m=20, copies=20,
                          "traffic": None}}
 
 
+def time_lm_head(ctx, binding, torch, dev, stream, n_rows, hidden, vocab, peak, reps=10):
+    """falcon_lm_head_argmax (Section 3.1, Eq. 6: the LM head applied to the nodes' features, greedy token only)
+    at the workload's shape, hidden = query heads x head_dim: two distinct random heads alternate (together more
+    than L2) in one CUDA graph, replayed; CUDA events on the launching stream.  Not part of the step."""
+    g = torch.Generator(device=dev)
+    g.manual_seed(11)
+    heads = [torch.randn(vocab, hidden, device=dev, generator=g).bfloat16() for _ in range(2)]
+    feat = torch.randn(n_rows, hidden, device=dev, generator=g).bfloat16()
+    out = torch.zeros(n_rows, dtype=torch.int32, device=dev)
+    calls = [binding.lm_argmax_args(n_rows, hidden, vocab, feat, hidden, w, hidden, out) for w in heads]
+    per_graph = 4 * len(calls)
+    with torch.cuda.stream(stream):
+        for a in calls:
+            ctx.falcon_lm_head_argmax(a)    # the first call sets the kernel's attributes: before the capture
+        stream.synchronize()
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr, stream=stream):
+            for _ in range(4):
+                for a in calls:
+                    ctx.falcon_lm_head_argmax(a)
+        for _ in range(3):
+            gr.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            gr.replay()
+        e1.record(stream)
+        stream.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (reps * per_graph)
+    nbytes = 2 * vocab * hidden + 2 * n_rows * hidden + 4 * n_rows
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"rows": n_rows, "hidden": hidden, "vocab": vocab, "us_per_call": us, "bytes_per_call": nbytes,
+            "useful_tflops": 2.0 * n_rows * hidden * vocab / (us * 1e-6) / 1e12,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                         "traffic": None}}
+
+
 # --------------------------------------------------------------------------- GPU arm
 ATTN_KERNELS = {"auto": 0, "simt": 1, "tc": 2, "tck": 3, "warp": 4}   # falcon.h FALCON_ATTN_*
 
@@ -445,6 +482,8 @@ def run_falcon(args):
 
     # ---------------- outside the step: the selection that grows the tree (the row next to the hot path) ----
     topm = time_topm(ctx, binding, torch, dev, stream, logits_h, peak) if world == 1 else None
+    lm = (time_lm_head(ctx, binding, torch, dev, stream, tb.total_nodes, spec.n_q_heads * spec.head_dim, spec.vocab, peak)
+          if world == 1 else None)
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -472,7 +511,7 @@ def run_falcon(args):
         "gpu_launches": args.steps * (NL + 2),
         "clocks": clocks,
         "cpu_baseline": cpu,
-        "extras": {"falcon_topm": topm},
+        "extras": {"falcon_topm": topm, "falcon_lm_head_argmax": lm},
         "wall_s_timed": t_wall,
     }
     print(json.dumps(line))

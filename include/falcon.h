@@ -214,7 +214,9 @@ int falcon_tree_accept(falcon_ctx* ctx, const falcon_accept_args* args, void* st
  *   max_out[i]    = that logit (optional)
  *
  * The head is a bias-free linear map stored row by row ([vocab, hidden], what the
- * LLaMA / Vicuna checkpoints hold).  falcon_tree_accept with logits == NULL then
+ * LLaMA / Vicuna checkpoints hold) and a constant: the kernel starts reading it
+ * while the previous kernel of the stream is still finishing, so that kernel must
+ * not be the one that writes lm_head.  falcon_tree_accept with logits == NULL then
  * finds the accepted path from argmax_out.  The sums are taken in fp32 in the
  * tensor core's order: two logits closer than that rounding may swap places
  * relative to an exact evaluation.

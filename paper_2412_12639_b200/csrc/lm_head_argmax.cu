@@ -11,9 +11,9 @@
 // hits after the first CTA).  tcgen05.mma with the nodes on the M side (128 per tile; up to two
 // tiles resident, so up to 256 nodes read the head once) and the CTA's vocabulary rows on the N
 // side (up to 256 per instruction) accumulates in TMEM; four warps then read one accumulator row
-// (= one node) each, 32 columns at a time, and keep the first maximum.  Per-CTA results go to
-// scratch and the last CTA to arrive folds them in vocabulary order, so ties go to the lowest
-// index whatever the timing.
+// (= one node) each, 32 columns at a time, and keep the first maximum.  A CTA's result for a node
+// is one 64-bit atomicMax on a word ordered by (logit, then lower index), so ties go to the lowest
+// index whatever the timing; the last CTA to arrive unpacks the words.
 //
 // Warp roles: 0 = TMA producer (one thread), 1 = MMA issuer (one elected thread) and TMEM owner,
 // 2-5 = accumulator readers.  Every wait is bounded; a wait that gives up sets FALCON_DEV_TIMEOUT
@@ -34,7 +34,7 @@ constexpr int kLmKC = 64;             // hidden columns per ring stage: one 128-
 constexpr int kLmMaxStages = 8;
 constexpr int kLmTileMax = 256;       // vocabulary rows per MMA (the N side) at most
 constexpr uint32_t kLmSmemMax = 232448;
-constexpr uint32_t kLmFeatTile = 128u * kLmKC * 2u;  // bytes of one 128-node x 64-column feature tile
+constexpr uint32_t kLmFeatPad = 64u * kLmKC * 2u;    // see f_rows: what a 64-row feature tile leaves for the MMA to read past
 
 enum LmBar {
   kLmBarFull = 0,                            // [kLmMaxStages] a stage's tiles have landed
@@ -44,11 +44,15 @@ enum LmBar {
   kLmBarDone,
   kLmNumBars
 };
-constexpr uint32_t kLmSmallBytes = 8u * kLmNumBars + 16u;  // barriers, TMEM base, abort flag, last-CTA flag
+constexpr uint32_t kLmSmallBytes = kLmFeatPad + 8u * kLmNumBars + 16u;  // pad, barriers, TMEM base, abort flag, last-CTA flag
 
 struct LmParams {
   int32_t n_rows, vocab;
-  int32_t n_kc;       // ring stages per accumulator tile = ceil(hidden / 64)
+  int32_t n_kc;       // 64-column chunks of the hidden dimension = ceil(hidden / 64)
+  int32_t kch;        // chunks per ring stage
+  int32_t f_rows;     // rows of a feature tile as loaded: 128, or with a single tile the number of nodes rounded up
+                      // to 8 (64 at least); the MMA still reads 128 rows, and what follows the tile gives
+                      // accumulator rows that nobody looks at
   int32_t n_mt;       // 128-node tiles
   int32_t m_res;      // node tiles resident in TMEM at once (1 or 2)
   int32_t tile_n;     // vocabulary rows per MMA (multiple of 16)
@@ -58,10 +62,20 @@ struct LmParams {
   int32_t* argmax_out;
   float* max_out;
   int32_t* status;
-  float* part_val;    // [n_rows, CTAs]
-  int32_t* part_idx;  // [n_rows, CTAs]
-  int* ticket;        // zero between calls
+  unsigned long long* best;  // [n_rows] the nodes' best (logit, index) so far as one orderable word; zero between calls
+  int* ticket;               // zero between calls
 };
+
+// (logit, index) as one word whose unsigned order is "larger logit first, then the lower index"; 0 = nothing.
+__device__ __forceinline__ unsigned long long lm_pack(float x, int idx) {
+  const uint32_t b = __float_as_uint(x + 0.f);  // -0 -> +0
+  const uint32_t key = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+  return (static_cast<unsigned long long>(key) << 32) | static_cast<uint32_t>(~idx);
+}
+__device__ __forceinline__ float lm_unpack_val(unsigned long long w) {
+  const uint32_t k = static_cast<uint32_t>(w >> 32);
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
 
 __device__ __forceinline__ bool lm_wait_drain(uint32_t bar, uint32_t parity) {
   for (uint32_t it = 0; it < (1u << 20); ++it) {
@@ -79,7 +93,7 @@ __global__ void __launch_bounds__(kLmThreads, 1)
 lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_f, const LmParams p) {
   extern __shared__ __align__(1024) unsigned char smem_gen[];
   const uint32_t smem_base = smem_u32(smem_gen);
-  unsigned char* small = smem_gen + static_cast<uint32_t>(p.n_stages) * p.stage_bytes;
+  unsigned char* small = smem_gen + static_cast<uint32_t>(p.n_stages) * p.stage_bytes + kLmFeatPad;
   const uint32_t bars = smem_u32(small);
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(small + 8 * kLmNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(small + 8 * kLmNumBars + 4);
@@ -93,7 +107,30 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
   const int n_vt = (v_hi - v_lo + p.tile_n - 1) / p.tile_n;  // >= 1 by construction of the grid
   const int n_groups = (p.n_mt + p.m_res - 1) / p.m_res;
   const uint32_t tmem_cols = static_cast<uint32_t>(p.m_res) * 256u;
-  const uint32_t w_bytes = static_cast<uint32_t>(p.tile_n) * (kLmKC * 2u);
+  const uint32_t w_bytes = static_cast<uint32_t>(p.tile_n) * (kLmKC * 2u);   // one chunk of the head tile
+  const uint32_t f_bytes = static_cast<uint32_t>(p.f_rows) * (kLmKC * 2u);   // one chunk of one feature tile
+  const int n_ks = (p.n_kc + p.kch - 1) / p.kch;                             // ring stages per accumulator tile
+  const int n_iter = n_groups * n_vt * n_ks;                                 // ring stages this CTA goes through
+  const int n_pre = min(S, n_iter);
+  // CTAs start at different places of the hidden dimension (a sum does not care where it starts), so that at
+  // any moment they read different column ranges of their rows instead of all the same one.
+  const int rot = static_cast<int>((static_cast<unsigned>(cta) * 11u) % static_cast<unsigned>(n_ks));
+  // Ring stage `it` = (node-tile group, vocabulary tile, K step), K fastest.  Its chunks are asked for back to
+  // back; a chunk past the hidden size reads as zeros, and so does a node tile past the last one.
+  auto issue_head = [&](int it) {
+    const int st = it % S, kq = (it % n_ks + rot) % n_ks, vt = (it / n_ks) % n_vt;
+    const uint32_t dst = smem_base + static_cast<uint32_t>(st) * p.stage_bytes;
+    for (int c = 0; c < p.kch; ++c)
+      tma_load_5d(dst + c * w_bytes, &tm_w, bar(kLmBarFull + st), (kq * p.kch + c) * kLmKC, v_lo + vt * p.tile_n, 0, 0, 0);
+  };
+  auto issue_feat = [&](int it) {
+    const int st = it % S, kq = (it % n_ks + rot) % n_ks, g = it / (n_ks * n_vt);
+    const uint32_t fdst = smem_base + static_cast<uint32_t>(st) * p.stage_bytes + static_cast<uint32_t>(p.kch) * w_bytes;
+    for (int c = 0; c < p.kch; ++c)
+      for (int j = 0; j < p.m_res; ++j)
+        tma_load_5d(fdst + (c * p.m_res + j) * f_bytes, &tm_f, bar(kLmBarFull + st), (kq * p.kch + c) * kLmKC,
+                    (g * p.m_res + j) * 128, 0, 0, 0);
+  };
 
   if (warp == 0) {
     if (lane == 0) {
@@ -103,6 +140,13 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
       prefetch_tmap(&tm_f);
       for (int i = 0; i < kLmNumBars; ++i) mbar_init(bar(i), i == kLmBarAccEmpty ? kLmReaders / 32 : 1);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      // The head is a constant of the model: its first ring fill is asked for before the wait below, while
+      // the previous kernel of the stream is still finishing.  The features are that kernel's to write.
+      if (!*abort_flag)
+        for (int it = 0; it < n_pre; ++it) {
+          mbar_expect_tx(bar(kLmBarFull + it), p.stage_bytes);
+          issue_head(it);
+        }
     }
     __syncwarp();
   } else if (warp == 1) {
@@ -122,22 +166,17 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
   if (warp == 0) {
     // ================================ TMA producer ================================
     if (lane == 0) {
-      int it = 0;
       bool ok = !*abort_flag;
-      for (int g = 0; ok && g < n_groups; ++g) {
-        for (int vt = 0; ok && vt < n_vt; ++vt) {
-          for (int kc = 0; ok && kc < p.n_kc; ++kc, ++it) {
-            const int st = it % S;
-            if (it >= S) ok = mbar_wait(bar(kLmBarEmpty + st), (it / S - 1) & 1, abort_flag);
-            if (!ok) break;
-            const uint32_t dst = smem_base + static_cast<uint32_t>(st) * p.stage_bytes;
-            mbar_expect_tx(bar(kLmBarFull + st), p.stage_bytes);
-            tma_load_5d(dst, &tm_w, bar(kLmBarFull + st), kc * kLmKC, v_lo + vt * p.tile_n, 0, 0, 0);
-            for (int j = 0; j < p.m_res; ++j)  // (a node tile past the last one reads as zeros)
-              tma_load_5d(dst + w_bytes + j * kLmFeatTile, &tm_f, bar(kLmBarFull + st), kc * kLmKC, (g * p.m_res + j) * 128, 0,
-                          0, 0);
-          }
-        }
+      int it = ok ? n_pre : 0;
+      if (ok)
+        for (int i = 0; i < n_pre; ++i) issue_feat(i);
+      for (; ok && it < n_iter; ++it) {
+        const int st = it % S;
+        ok = mbar_wait(bar(kLmBarEmpty + st), (it / S - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(bar(kLmBarFull + st), p.stage_bytes);
+        issue_head(it);
+        issue_feat(it);
       }
       if (!ok || *abort_flag) {
         // Some wait gave up.  The tiles asked for still arrive: stay until they have, so that no copy
@@ -156,20 +195,23 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
         if (tile > 0) ok = mbar_wait_warp(bar(kLmBarAccEmpty), (tile - 1) & 1, abort_flag);  // the readers are done with TMEM
         if (!ok) break;
         tc_fence_after();
-        for (int kc = 0; ok && kc < p.n_kc; ++kc, ++it) {
+        for (int ks = 0; ok && ks < n_ks; ++ks, ++it) {
           const int st = it % S;
           ok = mbar_wait_warp(bar(kLmBarFull + st), (it / S) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           if (elected) {
-            const uint32_t wbase = smem_base + static_cast<uint32_t>(st) * p.stage_bytes, fbase = wbase + w_bytes;
-            for (int j = 0; j < p.m_res; ++j) {
+            const uint32_t wbase = smem_base + static_cast<uint32_t>(st) * p.stage_bytes;
+            const uint32_t fbase = wbase + static_cast<uint32_t>(p.kch) * w_bytes;
+            for (int c = 0; c < p.kch; ++c) {
+              for (int j = 0; j < p.m_res; ++j) {
 #pragma unroll
-              for (int kk = 0; kk < kLmKC / 16; ++kk) {
-                // features (A) and head rows (B): both K-major, 16 hidden columns = 32 bytes inside the 128-byte swizzle row
-                const uint64_t ad = smem_desc(fbase + j * kLmFeatTile + kk * 32, 16, 1024);
-                const uint64_t bd = smem_desc(wbase + kk * 32, 16, 1024);
-                umma_bf16_ss(tmem_base + static_cast<uint32_t>(j) * 256u, ad, bd, p.idesc, (kc > 0 || kk > 0) ? 1u : 0u);
+                for (int kk = 0; kk < kLmKC / 16; ++kk) {
+                  // features (A) and head rows (B): both K-major, 16 hidden columns = 32 bytes inside the 128-byte swizzle row
+                  const uint64_t ad = smem_desc(fbase + (c * p.m_res + j) * f_bytes + kk * 32, 16, 1024);
+                  const uint64_t bd = smem_desc(wbase + c * w_bytes + kk * 32, 16, 1024);
+                  umma_bf16_ss(tmem_base + static_cast<uint32_t>(j) * 256u, ad, bd, p.idesc, (ks > 0 || c > 0 || kk > 0) ? 1u : 0u);
+                }
               }
             }
             umma_commit(bar(kLmBarEmpty + st));
@@ -227,10 +269,8 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         const int node = (g * p.m_res + j) * 128 + r;
-        if (j < p.m_res && node < p.n_rows) {
-          p.part_val[static_cast<int64_t>(node) * n_cta + cta] = ok ? best[j] : -INFINITY;
-          p.part_idx[static_cast<int64_t>(node) * n_cta + cta] = ok ? idx[j] : INT_MAX;
-        }
+        // one atomic per node and CTA: the order of arrival does not matter, the word's order decides
+        if (j < p.m_res && node < p.n_rows && ok && idx[j] != INT_MAX) atomicMax(p.best + node, lm_pack(best[j], idx[j]));
       }
     }
     // the last CTA to arrive folds the CTAs' results in vocabulary order
@@ -244,27 +284,10 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
     if (*s_last) {
       __threadfence();
       for (int node = rt; node < p.n_rows; node += kLmReaders) {
-        float bv = -INFINITY;
-        int bi = INT_MAX;
-        const int64_t o = static_cast<int64_t>(node) * n_cta;
-        for (int c = 0; c < n_cta; c += 8) {  // eight partials in flight: the loads are independent
-          float v[8];
-          int ix[8];
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const bool in = c + k < n_cta;
-            v[k] = in ? __ldcg(p.part_val + o + c + k) : -INFINITY;
-            ix[k] = in ? __ldcg(p.part_idx + o + c + k) : INT_MAX;
-          }
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            if (v[k] > bv) {  // CTAs ascend in vocabulary: strict keeps the lowest index
-              bv = v[k];
-              bi = ix[k];
-            }
-        }
-        p.argmax_out[node] = bi == INT_MAX ? 0 : bi;
-        if (p.max_out) p.max_out[node] = bv;
+        const unsigned long long w = __ldcg(p.best + node);
+        p.best[node] = 0ull;  // ready for the next call
+        p.argmax_out[node] = w ? static_cast<int>(~static_cast<uint32_t>(w)) : 0;
+        if (p.max_out) p.max_out[node] = w ? lm_unpack_val(w) : -INFINITY;
       }
       if (rt == 0) *p.ticket = 0;  // ready for the next call
     }
@@ -287,11 +310,20 @@ int launch_lm_head_argmax(falcon_ctx* ctx, const falcon_lm_argmax_args& a, cudaS
   int span = ((V + ctx->sm_count - 1) / ctx->sm_count + 15) & ~15;
   const int n_cta = (V + span - 1) / span;
   const int tile_n = span < kLmTileMax ? span : kLmTileMax;
-  const uint32_t stage_bytes = static_cast<uint32_t>(tile_n) * (kLmKC * 2u) + static_cast<uint32_t>(m_res) * kLmFeatTile;
+  const int f_rows = n_mt > 1 ? 128 : (N <= 64 ? 64 : ((N + 7) & ~7));
+  const int n_kc = (H + kLmKC - 1) / kLmKC;
+  // Chunks per stage: two where two such stages fit.  Fewer, larger stages mean fewer trips round the ring
+  // (32000 x 4096, 60 nodes: 43 us with two chunks in three stages against 53 with one in five and 46 with
+  // three in two; a head stored chunk by chunk so that a tile is contiguous made no difference).
+  const uint32_t chunk_bytes = (static_cast<uint32_t>(tile_n) + static_cast<uint32_t>(m_res * f_rows)) * (kLmKC * 2u);
+  int kch = (2 * 2 * chunk_bytes <= kLmSmemMax - kLmSmallBytes) ? 2 : 1;
+  if (kch > n_kc) kch = n_kc;
+  const uint32_t stage_bytes = static_cast<uint32_t>(kch) * chunk_bytes;
   int n_stages = static_cast<int>((kLmSmemMax - kLmSmallBytes) / stage_bytes);
   if (n_stages > kLmMaxStages) n_stages = kLmMaxStages;
   if (n_stages < 2) return FALCON_ERR_CAPACITY;
   const uint32_t smem_bytes = static_cast<uint32_t>(n_stages) * stage_bytes + kLmSmallBytes;
+
 
   if (!ctx->lm_attr_set) {
     cudaError_t e = cudaFuncSetAttribute(lm_head_argmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -299,10 +331,8 @@ int launch_lm_head_argmax(falcon_ctx* ctx, const falcon_lm_argmax_args& a, cudaS
     if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaFuncSetAttribute(lm_head_argmax_kernel)");
     ctx->lm_attr_set = true;
   }
-  const size_t part = static_cast<size_t>(N) * n_cta;
-  int rc = ensure_workspace(ctx, part * 8 + 256);
-  if (rc) return rc;
-  rc = ensure_tickets(ctx, 1, s);
+  // scratch that is zero between calls: the arrival counter and one 64-bit word per node
+  int rc = ensure_tickets(ctx, 2 + 2 * N, s);
   if (rc) return rc;
 
   // Tensor maps: [hidden, rows] with the hidden index contiguous; a box is 64 columns x the tile's
@@ -315,7 +345,7 @@ int launch_lm_head_argmax(falcon_ctx* ctx, const falcon_lm_argmax_args& a, cudaS
     const uint32_t w_box[5] = {kLmKC, static_cast<uint32_t>(tile_n), 1, 1, 1};
     const uint64_t f_dims[5] = {static_cast<uint64_t>(H), static_cast<uint64_t>(N), 1, 1, 1};
     const uint64_t f_strides[4] = {fs, fs * N, fs * N, fs * N};
-    const uint32_t f_box[5] = {kLmKC, 128, 1, 1, 1};
+    const uint32_t f_box[5] = {kLmKC, static_cast<uint32_t>(f_rows), 1, 1, 1};
     if (!get_tmap(ctx, a.lm_head, w_dims, w_strides, w_box, &mw) || !get_tmap(ctx, a.features, f_dims, f_strides, f_box, &mf)) {
       ctx->last_error = "cuTensorMapEncodeTiled failed";
       return FALCON_ERR_CUDA;
@@ -325,7 +355,9 @@ int launch_lm_head_argmax(falcon_ctx* ctx, const falcon_lm_argmax_args& a, cudaS
   LmParams p;
   p.n_rows = N;
   p.vocab = V;
-  p.n_kc = (H + kLmKC - 1) / kLmKC;
+  p.n_kc = n_kc;
+  p.kch = kch;
+  p.f_rows = f_rows;
   p.n_mt = n_mt;
   p.m_res = m_res;
   p.tile_n = tile_n;
@@ -336,9 +368,8 @@ int launch_lm_head_argmax(falcon_ctx* ctx, const falcon_lm_argmax_args& a, cudaS
   p.argmax_out = a.argmax_out;
   p.max_out = a.max_out;
   p.status = a.status;
-  p.part_val = static_cast<float*>(ctx->ws);
-  p.part_idx = reinterpret_cast<int32_t*>(static_cast<float*>(ctx->ws) + part);
   p.ticket = ctx->tickets;
+  p.best = reinterpret_cast<unsigned long long*>(ctx->tickets + 2);
 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_cta);

@@ -670,7 +670,7 @@ def test_lm_head_argmax_integer_data_is_bit_exact(N, Hd, V):
     f = synth.f32_to_bf16_bits(fi.astype(np.float32))
     w = synth.f32_to_bf16_bits(wi.astype(np.float32))
     g_ref, best_ref = oracle.lm_head_argmax(f, w)
-    for _ in range(2):                                         # twice: the arrival counter must come back to zero
+    for _ in range(2):                                         # twice: the scratch must come back to zero
         g, mx, status, rc = H.run_lm_argmax(f, w)
         assert rc == 0 and status == 0
         np.testing.assert_array_equal(g, g_ref)
@@ -685,6 +685,15 @@ def test_lm_head_argmax_random_data(N, Hd, V, pad):
     w = synth.normal_bf16(rng, (V, Hd + pad))
     g, g_ref = assert_lm_argmax(f, w, hidden=Hd)
     assert np.mean(g == g_ref) > 0.95                          # near-ties are rare with continuous data
+
+
+def test_lm_head_argmax_full_size_7b_shape():
+    # the size bench.py times: 60 nodes, hidden 4096, vocabulary 32000 (143 CTAs, 64 chunks of 64 columns each)
+    rng = np.random.default_rng(2024)
+    f = synth.normal_bf16(rng, (60, 4096))
+    w = synth.normal_bf16(rng, (32000, 4096), std=0.02)
+    g, g_ref = assert_lm_argmax(f, w)
+    assert np.mean(g == g_ref) > 0.95
 
 
 def test_lm_head_argmax_special_values():
@@ -798,8 +807,8 @@ def test_abi_rejects_bad_arguments_without_launching():
         == binding.ERR_INVALID_ARG
     assert c.falcon_tree_accept(binding.accept_args(dt.desc(), 10, lg, 10, g, path, 4, n, nxt), check=False) \
         == binding.ERR_INVALID_ARG
-    assert c.falcon_tree_accept(binding.accept_args(dt.desc(), 10, None, 10, g, path, 128, n, nxt), check=False) \
-        == binding.ERR_INVALID_ARG
+    assert c.falcon_tree_accept(binding.accept_args(dt.desc(), 10, lg, 10, None, path, 128, n, nxt), check=False) \
+        == binding.ERR_INVALID_ARG                             # (logits == NULL alone is legal: g is then an input)
     torch.cuda.synchronize()
 
 
