@@ -5,7 +5,7 @@
 // [N, V] fp32 result is never written: the argmax is taken where the accumulator is read.
 //
 // The head (V x hidden bf16, 262 MB at 32000 x 4096) is read once and dominates: the kernel is
-// bound by HBM, the tensor core is about a quarter busy.  Every CTA owns a run of vocabulary rows
+// bound by HBM, the tensor core is about a third busy.  Every CTA owns a run of vocabulary rows
 // (V split evenly over the SMs, in steps of 16, so one launch is one wave) and streams it through a
 // TMA ring in chunks of 64 hidden columns together with the matching chunk of the features (L2
 // hits after the first CTA).  tcgen05.mma with the nodes on the M side (128 per tile; up to two
