@@ -95,6 +95,24 @@ def argmax(logits, vocab=None, n_threads=0):
     return g
 
 
+def sample_tokens(logits, temperature, u, vocab=None, want_cdf=False, n_threads=0):
+    """logits: C-contiguous fp32 [N, stride]; u: fp32 [N] uniforms in [0, 1).  Returns g [N] int32 (and the
+    normalised partial sums [N, V] float64 with want_cdf)."""
+    assert logits.dtype == np.float32 and logits.ndim == 2 and logits.flags.c_contiguous
+    N, stride = logits.shape
+    V = stride if vocab is None else vocab
+    u = np.ascontiguousarray(u, dtype=np.float32)
+    assert u.shape == (N,)
+    g = np.empty(N, dtype=np.int32)
+    cdf = np.empty((N, V), dtype=np.float64) if want_cdf else None
+    rc = lib().oracle_sample_tokens(_p(logits, C.c_float), C.c_int32(N), C.c_int32(V), C.c_int64(stride),
+                                    C.c_double(temperature), _p(u, C.c_float), _p(g, C.c_int32),
+                                    _p(cdf, C.c_double) if want_cdf else None, C.c_int(n_threads))
+    if rc:
+        raise ValueError("oracle_sample_tokens failed: %d" % rc)
+    return (g, cdf) if want_cdf else g
+
+
 def lm_head_argmax(feat_bits, head_bits, hidden=None, want_logits=False, n_threads=0):
     """feat_bits: uint16 (bf16 bit patterns) [N, feat_stride]; head_bits: uint16 [V, head_stride]; the first
     `hidden` columns of both are used.  Returns (g [N] int32, best [N] float64[, logits [N, V] float64])."""

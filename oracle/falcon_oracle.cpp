@@ -254,6 +254,64 @@ int oracle_argmax(const float* logits, int32_t N, int32_t V, int64_t stride, int
   return 0;
 }
 
+// The target model's own token at every node when decoding is not greedy.  Section 3.1: the LM
+// head gives "the probability distribution ..., from which the next token is sampled"; Appendix A
+// only says that in a non-greedy setting the drafted children are sampled, and Section 3.4 that
+// verification is "consistent with SpecInfer" - the paper states no acceptance rule of its own.
+// The reading taken here is the simplest lossless one: at every node the target draws its token
+// from softmax(logits / temperature), and a drafted child is accepted when it carries that token
+// (with temperature -> 0 this is the greedy rule).  The draw is the inverse-CDF one, with the
+// uniform number u[i] in [0, 1) supplied by the caller:
+//   w_v = exp((logits[i, v] - max_v logits[i, v]) / temperature)   (a NaN logit has weight 0),
+//   g[i] = the lowest v with  sum_{k <= v} w_k  >  u[i] * sum_k w_k,
+// sums in vocabulary order, in double; if rounding leaves no such v, the last v with w_v > 0; a row
+// with no finite maximum (all NaN or -inf) gives 0.  cdf (optional, [N, V] doubles) receives the
+// normalised partial sums.  The accepted path then follows from g exactly as in the greedy case.
+int oracle_sample_tokens(const float* logits, int32_t N, int32_t V, int64_t stride, double temperature, const float* u,
+                         int32_t* g, double* cdf, int n_threads) {
+  if (N < 0 || V < 1 || stride < V || !(temperature > 0.0)) return 1;
+  const int nt = pick_threads(n_threads);
+  (void)nt;
+#pragma omp parallel for num_threads(nt)
+  for (int32_t i = 0; i < N; ++i) {
+    const float* row = logits + static_cast<int64_t>(i) * stride;
+    double top = -std::numeric_limits<double>::infinity();
+    for (int32_t v = 0; v < V; ++v)
+      if (static_cast<double>(row[v]) > top) top = row[v];
+    if (!std::isfinite(top)) {  // nothing to draw from (or a +inf logit, which takes everything: its first position)
+      int32_t idx = 0;
+      if (top > 0)
+        for (int32_t v = 0; v < V; ++v)
+          if (static_cast<double>(row[v]) == top) {
+            idx = v;
+            break;
+          }
+      g[i] = idx;
+      if (cdf)
+        for (int32_t v = 0; v < V; ++v) cdf[static_cast<int64_t>(i) * V + v] = v >= idx ? 1.0 : 0.0;
+      continue;
+    }
+    double total = 0.0;
+    for (int32_t v = 0; v < V; ++v) {
+      const double x = row[v];
+      if (x == x) total += std::exp((x - top) / temperature);
+    }
+    const double target = static_cast<double>(u[i]) * total;
+    double run = 0.0;
+    int32_t idx = -1, last = 0;
+    for (int32_t v = 0; v < V; ++v) {
+      const double x = row[v];
+      const double w = (x == x) ? std::exp((x - top) / temperature) : 0.0;
+      run += w;
+      if (w > 0.0) last = v;
+      if (idx < 0 && run > target) idx = v;
+      if (cdf) cdf[static_cast<int64_t>(i) * V + v] = run / total;
+    }
+    g[i] = idx >= 0 ? idx : last;
+  }
+  return 0;
+}
+
 // LM-head logits of the tree's nodes and their greedy argmax without a logits matrix in
 // between.  The verification pass ends in the target model's LM head: "the LM Head computes
 // the probability distribution based on the aggregated features" (Section 3.1) and Eq. 6 writes

@@ -709,3 +709,64 @@ def test_lm_head_argmax_agrees_with_the_logits_scan():
     srt = np.sort(logits, axis=1)
     assert np.all(srt[:, -1] - srt[:, -2] > 1e-3)
     assert np.array_equal(g, oracle.argmax(np.ascontiguousarray(logits.astype(np.float32))))
+
+
+# --------------------------------------------------------------------------- non-greedy token draw (Section 3.1)
+def test_sample_tokens_hand_worked():
+    c = GOLD["sample_tokens_basic"]
+    u = np.array(c["uniform_u"], dtype=np.float32)
+    lg = np.zeros((len(u), c["uniform_vocab"]), dtype=np.float32)
+    assert oracle.sample_tokens(lg, 1.0, u).tolist() == c["uniform_expected"]
+    assert oracle.sample_tokens(lg + 3.5, 0.7, u).tolist() == c["uniform_expected"]     # equal logits: any shift, any temperature
+    ub = np.array(c["b_u"], dtype=np.float32)
+    lb = np.tile(np.array(c["b_logits"], dtype=np.float32), (len(ub), 1))
+    assert oracle.sample_tokens(lb, c["b_temperature"], ub).tolist() == c["b_expected"]
+
+
+def test_sample_tokens_is_the_inverse_cdf_of_the_softmax():
+    rng = np.random.default_rng(8)
+    N, V, T = 40, 300, 1.7
+    lg = (2.0 * rng.standard_normal((N, V))).astype(np.float32)
+    u = rng.random(N).astype(np.float32)
+    g, cdf = oracle.sample_tokens(lg, T, u, want_cdf=True)
+    z = lg.astype(np.float64) / T
+    p = np.exp(z - z.max(axis=1, keepdims=True))
+    ref_cdf = np.cumsum(p, axis=1) / p.sum(axis=1, keepdims=True)      # numpy's softmax partial sums
+    assert np.allclose(cdf, ref_cdf, rtol=1e-12, atol=1e-15)
+    assert np.all(np.diff(cdf, axis=1) >= 0) and np.allclose(cdf[:, -1], 1.0)
+    ref = np.array([np.searchsorted(ref_cdf[i], u[i], side="right") for i in range(N)])
+    assert np.min(np.abs(ref_cdf - u[:, None].astype(np.float64))) > 1e-9   # no draw sits on a boundary
+    assert np.array_equal(g, ref)
+    assert np.array_equal(oracle.sample_tokens(lg + 11.0, T, u), g)    # softmax ignores a shift of the logits
+
+
+def test_sample_tokens_frequencies_follow_the_probabilities():
+    rng = np.random.default_rng(9)
+    V, T, draws = 6, 2.0, 40000
+    row = np.array([0.3, -1.0, 2.2, 0.0, 1.1, -3.0], dtype=np.float32)
+    p = np.exp(row.astype(np.float64) / T)
+    p /= p.sum()
+    g = oracle.sample_tokens(np.tile(row, (draws, 1)), T, rng.random(draws).astype(np.float32))
+    freq = np.bincount(g, minlength=V) / draws
+    assert np.all(np.abs(freq - p) < 5.0 * np.sqrt(p * (1 - p) / draws))
+
+
+def test_sample_tokens_limits_and_special_values():
+    rng = np.random.default_rng(10)
+    N, V = 25, 500
+    lg = rng.standard_normal((N, V)).astype(np.float32)
+    lg[np.arange(N), rng.integers(0, V, N)] += 3.0                      # a clear maximum per row
+    u = rng.random(N).astype(np.float32)
+    assert np.array_equal(oracle.sample_tokens(lg, 1e-3, u), oracle.argmax(lg))   # temperature -> 0: the greedy token
+    one = np.full((4, 50), -np.inf, dtype=np.float32)
+    one[np.arange(4), [7, 0, 49, 20]] = [1.0, -2.0, 0.5, 30.0]
+    for uu in (0.0, 0.5, 0.999):                                        # a single possible token: it is drawn
+        assert oracle.sample_tokens(one, 1.0, np.full(4, uu, np.float32)).tolist() == [7, 0, 49, 20]
+    nan = lg.copy()
+    g0 = oracle.sample_tokens(lg, 1.0, u)
+    nan[np.arange(N), g0] = np.nan                                      # the drawn token becomes impossible
+    g1 = oracle.sample_tokens(nan, 1.0, u)
+    assert np.all(g1 != g0)
+    assert np.all(oracle.sample_tokens(np.full((3, 9), np.nan, np.float32), 1.0, np.full(3, 0.4, np.float32)) == 0)
+    pad = np.concatenate([lg, np.full((N, 12), 80.0, np.float32)], axis=1)   # beyond `vocab`: never read
+    assert np.array_equal(oracle.sample_tokens(np.ascontiguousarray(pad), 1.0, u, vocab=V), g0)
