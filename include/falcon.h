@@ -184,6 +184,19 @@ int falcon_tree_attn_kernel(falcon_ctx* ctx, const falcon_attn_args* args);
  *   path[b]   = its root-to-node chain (local indices, path[b][0] == 0, rest -1)
  *   n_path[b] = nodes on the path (accepted drafted tokens = n_path - 1)
  *   next_token[b] = g[last node of the path]
+ *
+ * Non-greedy decoding (temperature > 0).  Section 3.1: the LM head gives the
+ * probability distribution "from which the next token is sampled"; the paper
+ * states no acceptance rule for this case (Appendix A only says the drafted
+ * children are sampled; Section 3.4 that verification follows SpecInfer).  The
+ * rule here is the simplest one that leaves the output distribution the target's
+ * own: at every node the target draws its token and a drafted child is accepted
+ * when it carries that token.  The draw is the inverse-CDF one with the caller's
+ * uniform number: w_v = exp((logits[i,v] - max) / temperature) (NaN: weight 0),
+ * g[i] = lowest v with sum_{k<=v} w_k > uniforms[i] * sum_k w_k (fp32 sums: a
+ * draw within rounding of a boundary may fall on either side; a row with no
+ * finite maximum gives 0, a +inf logit its first position).  Everything after g
+ * is as above.  vocab <= 262144 in this mode.
  * ------------------------------------------------------------------------- */
 typedef struct {
   falcon_tree_desc tree;
@@ -197,6 +210,10 @@ typedef struct {
   int32_t path_stride;    /* >= max_tree                                              */
   int32_t* n_path;        /* [B]                                                      */
   int32_t* next_token;    /* [B]                                                      */
+  float temperature;      /* 0: greedy, g = the argmax (the paper's setting).  > 0:   */
+                          /* non-greedy, g[i] is the target's own draw from           */
+                          /* softmax(logits[i] / temperature), see below              */
+  const float* uniforms;  /* [N] in [0, 1), one per node; read when temperature > 0   */
 } falcon_accept_args;
 
 int falcon_tree_accept(falcon_ctx* ctx, const falcon_accept_args* args, void* stream);

@@ -48,7 +48,8 @@ class AttnArgs(C.Structure):
 class AcceptArgs(C.Structure):
     _fields_ = [("tree", TreeDesc), ("vocab", C.c_int32), ("logits_stride", C.c_int64), ("logits", C.c_void_p),
                 ("argmax_out", C.c_void_p), ("path", C.c_void_p), ("path_stride", C.c_int32),
-                ("n_path", C.c_void_p), ("next_token", C.c_void_p)]
+                ("n_path", C.c_void_p), ("next_token", C.c_void_p), ("temperature", C.c_float),
+                ("uniforms", C.c_void_p)]
 
 
 class TopmArgs(C.Structure):
@@ -243,9 +244,10 @@ def attn_args(tree: TreeDesc, n_q_heads, n_kv_heads, head_dim, sm_scale, q, out,
 
 
 def accept_args(tree: TreeDesc, vocab, logits, logits_stride, argmax_out, path, path_stride, n_path,
-                next_token) -> AcceptArgs:
+                next_token, temperature: float = 0.0, uniforms=None) -> AcceptArgs:
+    """temperature > 0: the nodes' tokens are drawn from softmax(logits / temperature) with `uniforms` [N]."""
     return AcceptArgs(tree, vocab, logits_stride, _ptr(logits), _ptr(argmax_out), _ptr(path), path_stride,
-                      _ptr(n_path), _ptr(next_token))
+                      _ptr(n_path), _ptr(next_token), temperature, _ptr(uniforms))
 
 
 def topm_args(n_rows, vocab, logits, logits_stride, m, top_val, top_idx) -> TopmArgs:

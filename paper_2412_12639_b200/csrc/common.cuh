@@ -50,6 +50,7 @@ int launch_feature_gather(falcon_ctx* ctx, const falcon_gather_args& a, cudaStre
 int check_gather_args(const falcon_gather_args& g, int max_tree);
 int launch_tree_topm(falcon_ctx* ctx, const falcon_topm_args& a, cudaStream_t s);
 int launch_tree_search(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_t s);
+int launch_tree_sample(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_t s);
 int launch_lm_head_argmax(falcon_ctx* ctx, const falcon_lm_argmax_args& a, cudaStream_t s);
 int launch_tree_attn_simt(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s);
 int launch_tree_attn_tc(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s);

@@ -191,9 +191,17 @@ int falcon_tree_accept(falcon_ctx* ctx, const falcon_accept_args* a, void* strea
   if (rc) return rc;
   if (!a->argmax_out || !a->path || !a->n_path || !a->next_token) return FALCON_ERR_INVALID_ARG;
   if (a->path_stride < a->tree.max_tree) return FALCON_ERR_INVALID_ARG;
-  if (!a->logits) return launch_tree_search(ctx, *a, static_cast<cudaStream_t>(stream));  // g is given
+  if (!(a->temperature >= 0.f)) return FALCON_ERR_INVALID_ARG;
+  if (!a->logits) {  // g is given
+    if (a->temperature != 0.f) return FALCON_ERR_INVALID_ARG;
+    return launch_tree_search(ctx, *a, static_cast<cudaStream_t>(stream));
+  }
   if (a->vocab < 1 || a->logits_stride < a->vocab) return FALCON_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(a->logits) & 3) return FALCON_ERR_INVALID_ARG;
+  if (a->temperature > 0.f) {
+    if (!a->uniforms || (reinterpret_cast<uintptr_t>(a->uniforms) & 3)) return FALCON_ERR_INVALID_ARG;
+    return launch_tree_sample(ctx, *a, static_cast<cudaStream_t>(stream));
+  }
   return launch_tree_accept(ctx, *a, static_cast<cudaStream_t>(stream));
 }
 

@@ -28,6 +28,11 @@ struct AcceptParams {
   float* part_val;  // [N, chunks]
   int32_t* part_idx;
   int* tickets;     // [B]
+  // non-greedy only
+  float inv_t_log2e;       // log2(e) / temperature
+  const float* uniforms;   // [N]
+  float* part_sum;         // [N, chunks] sum of exp((x - chunk max) / temperature)
+  int* row_tickets;        // [N]
 };
 
 struct Best {
@@ -208,6 +213,237 @@ __global__ void __launch_bounds__(kAcceptThreads) tree_search_kernel(const Accep
   search_tree(p, b, base, T_real, g, s_par, s_tok, s_g, s_key);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Non-greedy acceptance: g[i] is the target's own draw from softmax(logits[i] / temperature)
+// (Section 3.1: the next token is sampled from the LM head's distribution) by the inverse-CDF rule
+// with the caller's uniform u[i]: the lowest v whose partial sum of weights exceeds u[i] times the
+// total.  One launch.  Every CTA takes one chunk (at most 4096 entries, in registers) of one row:
+// chunk maximum, then the chunk's sum of weights relative to it.  The last CTA of a row to finish
+// (counter) rescales the chunks' sums to the row maximum, finds the chunk in which the partial sums
+// pass the target, loads that chunk again (L2) and finds the position: warp by warp, then row of
+// 32 by row, then by a scan over the lanes.  The last row of a sequence (second counter) runs the
+// same path search as the greedy call.  fp32 sums: a draw within rounding of a boundary between
+// two tokens may fall on either side.
+constexpr int kSamplePerLane = 16;
+constexpr int kSampleChunkMax = (kAcceptThreads / 32) * 32 * kSamplePerLane;  // 4096
+
+__device__ __forceinline__ float warp_add(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__global__ void __launch_bounds__(kAcceptThreads) tree_sample_kernel(const AcceptParams p) {
+  constexpr int kWarps = kAcceptThreads / 32;
+  __shared__ Best warp_best[kWarps];
+  __shared__ float s_wsum[kWarps];
+  __shared__ float s_scaled[64];
+  __shared__ float s_bcast[4];
+  __shared__ int s_ibcast[4];
+  __shared__ int s_flag;
+  __shared__ int s_par[FALCON_T_MAX], s_tok[FALCON_T_MAX], s_g[FALCON_T_MAX];
+  __shared__ int s_key[kWarps];
+
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int row = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const float* rowp = p.logits + static_cast<int64_t>(row) * p.logits_stride;
+  int lo = 0, hi = p.batch;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (p.node_off[mid] <= row) lo = mid; else hi = mid;
+  }
+  const int b = lo;
+  const int base = p.node_off[b];
+  const int T_real = p.node_off[b + 1] - base;
+  const float kq = p.inv_t_log2e;
+
+  // entry k of lane l of warp w is element w * 512 + k * 32 + l of the chunk (coalesced rows of 32)
+  auto load_chunk = [&](int ch, float (&x)[kSamplePerLane], bool streaming) {
+    const int c0 = ch * p.chunk_len;
+    const int n = min(p.vocab, c0 + p.chunk_len) - c0;
+#pragma unroll
+    for (int k = 0; k < kSamplePerLane; ++k) {
+      const int j = warp * (32 * kSamplePerLane) + k * 32 + lane;
+      x[k] = j < n ? (streaming ? __ldcs(rowp + c0 + j) : __ldcg(rowp + c0 + j)) : __int_as_float(0x7fc00000);  // NaN = no entry
+    }
+    return c0;
+  };
+
+  // ---- every CTA: the chunk's maximum (and where it first occurs) and its sum of weights ----
+  {
+    float x[kSamplePerLane];
+    const int c0 = load_chunk(chunk, x, true);
+    Best mine{-INFINITY, kNone};
+#pragma unroll
+    for (int k = 0; k < kSamplePerLane; ++k) take(mine, x[k], c0 + warp * (32 * kSamplePerLane) + k * 32 + lane);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      Best other{__shfl_xor_sync(0xffffffffu, mine.v, o), __shfl_xor_sync(0xffffffffu, mine.i, o)};
+      mine = merge(mine, other);
+    }
+    if (lane == 0) warp_best[warp] = mine;
+    __syncthreads();
+    Best r = warp_best[0];
+#pragma unroll
+    for (int w = 1; w < kWarps; ++w) r = merge(r, warp_best[w]);
+    float s = 0.f;
+    if (r.v > -INFINITY && r.v < INFINITY) {
+#pragma unroll
+      for (int k = 0; k < kSamplePerLane; ++k)
+        if (x[k] == x[k]) s += exp2f((x[k] - r.v) * kq);
+    }
+    s = warp_add(s);
+    if (lane == 0) s_wsum[warp] = s;
+    __syncthreads();
+    if (tid == 0) {
+      float tot = 0.f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) tot += s_wsum[w];
+      const int64_t o = static_cast<int64_t>(row) * p.chunks + chunk;
+      p.part_val[o] = r.v;
+      p.part_sum[o] = tot;
+      p.part_idx[o] = r.i;
+      __threadfence();
+      s_flag = (atomicAdd(&p.row_tickets[row], 1) == p.chunks - 1);
+    }
+    __syncthreads();
+    if (!s_flag) return;
+    __threadfence();
+  }
+
+  // ---- last CTA of the row: the chunk in which the partial sums pass u * total ----
+  if (tid == 0) {
+    const int64_t o = static_cast<int64_t>(row) * p.chunks;
+    float M = -INFINITY;
+    for (int c = 0; c < p.chunks; ++c) M = fmaxf(M, __ldcg(p.part_val + o + c));
+    int direct = -1, cstar = 0;
+    float resid = 0.f;
+    if (!(M > -INFINITY)) {
+      direct = 0;  // nothing to draw from
+    } else if (!(M < INFINITY)) {
+      for (int c = 0; c < p.chunks && direct < 0; ++c)  // a +inf logit takes everything: its first position
+        if (__ldcg(p.part_val + o + c) == M) direct = __ldcg(p.part_idx + o + c);
+    } else {
+      float total = 0.f;
+      for (int c = 0; c < p.chunks; ++c) {
+        const float mc = __ldcg(p.part_val + o + c);
+        const float sc = mc > -INFINITY ? __ldcg(p.part_sum + o + c) * exp2f((mc - M) * kq) : 0.f;
+        s_scaled[c] = sc;
+        total += sc;
+      }
+      const float target = p.uniforms[row] * total;
+      float run = 0.f;
+      int last = 0;
+      cstar = -1;
+      for (int c = 0; c < p.chunks; ++c) {
+        const float sc = s_scaled[c];
+        if (sc > 0.f) last = c;
+        if (run + sc > target) {
+          cstar = c;
+          break;
+        }
+        run += sc;
+      }
+      if (cstar < 0) {  // rounding left the target at or past the total: the end of the last chunk that has weight
+        cstar = last;
+        run -= s_scaled[last];
+      }
+      resid = target - run;
+    }
+    s_ibcast[0] = direct;
+    s_ibcast[1] = cstar;
+    s_bcast[0] = resid;
+    s_bcast[1] = M;
+    p.row_tickets[row] = 0;  // ready for the next call
+  }
+  __syncthreads();
+  int g = s_ibcast[0];
+  if (g < 0) {
+    // ---- the position inside that chunk: warp, then row of 32, then lane ----
+    const int cstar = s_ibcast[1];
+    const float M = s_bcast[1];
+    float x[kSamplePerLane], w[kSamplePerLane];
+    const int c0 = load_chunk(cstar, x, false);
+    float ws = 0.f;
+#pragma unroll
+    for (int k = 0; k < kSamplePerLane; ++k) {
+      w[k] = (x[k] == x[k]) ? exp2f((x[k] - M) * kq) : 0.f;
+      ws += w[k];
+    }
+    ws = warp_add(ws);
+    if (lane == 0) s_wsum[warp] = ws;
+    __syncthreads();
+    // every thread: which warp (the sums are the same in all of them)
+    float resid = s_bcast[0], tot = 0.f;
+#pragma unroll
+    for (int i = 0; i < kWarps; ++i) tot += s_wsum[i];
+    resid = fminf(resid, tot * 0.99999f);  // recomputed with the row maximum the chunk may sum to a hair less
+    int wstar = -1, wlast = 0;
+    float run = 0.f;
+#pragma unroll
+    for (int i = 0; i < kWarps; ++i) {
+      const float v = s_wsum[i];
+      if (v > 0.f) wlast = i;
+      if (wstar < 0) {
+        if (run + v > resid) wstar = i; else run += v;
+      }
+    }
+    if (wstar < 0) {
+      wstar = wlast;
+      run -= s_wsum[wlast];
+    }
+    if (warp == wstar) {
+      float rw = fminf(resid - run, s_wsum[wstar] * 0.99999f);
+      int kstar = -1, klast = 0;
+      float wk = 0.f, before = 0.f, acc = 0.f;
+#pragma unroll
+      for (int k = 0; k < kSamplePerLane; ++k) {
+        const float rs = warp_add(w[k]);
+        if (rs > 0.f) klast = k;
+        if (kstar < 0) {
+          if (acc + rs > rw) {
+            kstar = k;
+            before = acc;
+          } else {
+            acc += rs;
+          }
+        }
+      }
+      if (kstar < 0) kstar = klast;
+#pragma unroll
+      for (int k = 0; k < kSamplePerLane; ++k)
+        if (k == kstar) wk = w[k];
+      const float rsel = warp_add(wk);  // (if no row passed the target, `before` is 0 and the clamp below ends the search
+                                        // at the last entry of the last row that has weight)
+      float incl = wk;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const float t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      const float rl = fminf(rw - before, rsel * 0.99999f);
+      const unsigned pass = __ballot_sync(0xffffffffu, wk > 0.f && incl > rl);
+      const unsigned any = __ballot_sync(0xffffffffu, wk > 0.f);
+      const int lstar = pass ? __ffs(static_cast<int>(pass)) - 1 : (any ? 31 - __clz(static_cast<int>(any)) : 0);
+      if (lane == 0) s_ibcast[2] = c0 + wstar * (32 * kSamplePerLane) + kstar * 32 + lstar;
+    }
+    __syncthreads();
+    g = s_ibcast[2];
+  }
+  if (tid == 0) {
+    p.argmax_out[row] = g;
+    __threadfence();
+    s_flag = (atomicAdd(&p.tickets[b], 1) == T_real - 1);
+  }
+  __syncthreads();
+  if (!s_flag) return;
+  __threadfence();
+  // ---- last row of sequence b: the path search on the drawn tokens ----
+  const int gt = tid < min(T_real, FALCON_T_MAX) ? __ldcg(p.argmax_out + base + tid) : 0;
+  search_tree(p, b, base, T_real, gt, s_par, s_tok, s_g, s_key);
+  if (tid == 0) p.tickets[b] = 0;  // ready for the next call
+}
+
 constexpr int kAcceptMaxChunks = 64;  // vocabulary chunks per row at most (the static scratch is sized by it)
 
 // How a launch splits the vocabulary: enough CTAs for a few waves, chunks of at least 2048 elements
@@ -247,6 +483,10 @@ AcceptParams accept_params(const falcon_accept_args& a, int chunks, int chunk_le
   p.part_val = static_cast<float*>(part);
   p.part_idx = reinterpret_cast<int32_t*>(part) + static_cast<size_t>(a.tree.total_nodes) * chunks;
   p.tickets = tickets;
+  p.inv_t_log2e = 0.f;
+  p.uniforms = nullptr;
+  p.part_sum = nullptr;
+  p.row_tickets = nullptr;
   return p;
 }
 
@@ -276,6 +516,43 @@ int launch_tree_accept(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_
   cfg.numAttrs = 1;
   cudaError_t e = cudaLaunchKernelEx(&cfg, tree_accept_kernel, p);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "tree_accept_kernel launch");
+  return FALCON_OK;
+}
+
+// temperature > 0: the nodes' tokens are drawn instead of taken at the maximum.
+int launch_tree_sample(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_t s) {
+  const int N = a.tree.total_nodes, B = a.tree.batch;
+  if (N > 65535) return FALCON_ERR_CAPACITY;
+  int chunks, chunk_len;
+  accept_plan(ctx->sm_count, N, a.vocab, &chunks, &chunk_len);
+  const int min_chunks = (a.vocab + kSampleChunkMax - 1) / kSampleChunkMax;  // a chunk is held in registers
+  if (chunks < min_chunks) chunks = min_chunks;
+  if (chunks > kAcceptMaxChunks) return FALCON_ERR_CAPACITY;
+  chunk_len = ((a.vocab + chunks - 1) / chunks + 3) & ~3;
+  chunks = (a.vocab + chunk_len - 1) / chunk_len;
+
+  const size_t part = static_cast<size_t>(N) * chunks;
+  int rc = ensure_workspace(ctx, part * 12 + 256);
+  if (rc) return rc;
+  rc = ensure_tickets(ctx, static_cast<size_t>(B) + N, s);
+  if (rc) return rc;
+  AcceptParams p = accept_params(a, chunks, chunk_len, ctx->ws, ctx->tickets);
+  p.part_sum = reinterpret_cast<float*>(p.part_idx + part);
+  p.row_tickets = ctx->tickets + B;
+  p.uniforms = a.uniforms;
+  p.inv_t_log2e = kLog2e / a.temperature;
+
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(chunks, N);
+  cfg.blockDim = dim3(kAcceptThreads);
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, tree_sample_kernel, p);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "tree_sample_kernel launch");
   return FALCON_OK;
 }
 
@@ -362,6 +639,7 @@ extern "C" int falcon_tree_accept_static(const falcon_accept_args* a, void* stre
   if (a->vocab < 1 || a->logits_stride < a->vocab) return FALCON_ERR_INVALID_ARG;
   if (a->path_stride < a->tree.max_tree) return FALCON_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(a->logits) & 3) return FALCON_ERR_INVALID_ARG;
+  if (a->temperature != 0.f) return FALCON_ERR_UNSUPPORTED;  // the fixed scratch is sized for the greedy call
   // sizes beyond the fixed scratch are refused, never truncated
   if (a->tree.total_nodes > kStaticMaxNodes || a->tree.batch > kStaticMaxBatch) return FALCON_ERR_CAPACITY;
 

@@ -120,16 +120,18 @@ def assert_attn_close(out_bits, ref, node_off, report=False):
     return max_abs, rel
 
 
-def run_accept(dt: DevTrees, logits: np.ndarray, vocab=None, path_stride=128):
-    """logits fp32 [N, stride] -> (g, path, n_path, next_token) numpy."""
+def run_accept(dt: DevTrees, logits: np.ndarray, vocab=None, path_stride=128, temperature=0.0, uniforms=None):
+    """logits fp32 [N, stride] -> (g, path, n_path, next_token) numpy.  temperature > 0: the non-greedy call
+    with uniforms fp32 [N]."""
     ld = torch.from_numpy(np.ascontiguousarray(logits)).cuda()
+    ud = None if uniforms is None else torch.from_numpy(np.ascontiguousarray(uniforms, dtype=np.float32)).cuda()
     N, B = dt.host.total_nodes, dt.host.batch
     g = torch.full((N,), -7, dtype=torch.int32, device="cuda")
     path = torch.full((B, path_stride), -7, dtype=torch.int32, device="cuda")
     n_path = torch.full((B,), -7, dtype=torch.int32, device="cuda")
     nxt = torch.full((B,), -7, dtype=torch.int32, device="cuda")
     a = binding.accept_args(dt.desc(), logits.shape[1] if vocab is None else vocab, ld, logits.shape[1], g, path,
-                            path_stride, n_path, nxt)
+                            path_stride, n_path, nxt, temperature=temperature, uniforms=ud)
     ctx().falcon_tree_accept(a)
     torch.cuda.synchronize()
     return g.cpu().numpy(), path.cpu().numpy(), n_path.cpu().numpy(), nxt.cpu().numpy()

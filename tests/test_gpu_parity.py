@@ -636,6 +636,111 @@ def test_topm_rejects_bad_arguments_without_launching():
     assert (idx.cpu().numpy() == -7).all() and (val.cpu().numpy() == 3.0).all()
 
 
+# ------------------------------------------------------------------------ non-greedy acceptance (Section 3.1)
+SAMPLE_TOL = 1e-4   # fp32 partial sums of up to 32000 weights against the oracle's double ones, relative to the total
+
+
+def assert_valid_draws(lg, vocab, T, u, g):
+    """The kernel's token must be a valid inverse-CDF draw within fp32 rounding: the oracle's normalised partial
+    sums just before and at the token bracket u up to SAMPLE_TOL, and the token has weight."""
+    g_ref, cdf = oracle.sample_tokens(lg, T, u, vocab=vocab, want_cdf=True)
+    N = len(g)
+    assert g.min() >= 0 and g.max() < vocab
+    hi = cdf[np.arange(N), g]
+    lo = np.where(g > 0, cdf[np.arange(N), np.maximum(g - 1, 0)], 0.0)
+    assert np.all(hi - lo > 0), "a token without weight was drawn"
+    uu = u.astype(np.float64)
+    assert np.all(lo <= uu + SAMPLE_TOL) and np.all(uu < hi + SAMPLE_TOL), (np.max(lo - uu), np.max(uu - hi))
+    return g_ref
+
+
+@pytest.mark.parametrize("name", ["tiny", "v7b", "l13b", "ragged"])
+@pytest.mark.parametrize("T", [0.7, 1.0, 2.5])
+def test_sample_accept_on_the_workloads(name, T):
+    wl = synth.make_workload(name, with_logits=True)
+    tb = wl.trees
+    rng = np.random.default_rng(int(T * 10) + len(name))
+    u = rng.random(tb.total_nodes).astype(np.float32)
+    dt = H.DevTrees(tb)
+    for _ in range(2):                                         # twice: both counters must come back to zero
+        g, path, n_path, nxt = H.run_accept(dt, wl.logits, temperature=T, uniforms=u)
+        g_ref = assert_valid_draws(wl.logits, wl.logits.shape[1], T, u, g)
+        assert np.mean(g == g_ref) > 0.98
+        rp, rn, rt = oracle.tree_accept(tb.node_off, tb.parent, tb.token, g)   # the search, given the drawn tokens
+        np.testing.assert_array_equal(path, rp)
+        np.testing.assert_array_equal(n_path, rn)
+        np.testing.assert_array_equal(nxt, rt)
+
+
+@pytest.mark.parametrize("V,stride", [(8192, 8192), (32000, 32000), (1000, 1003), (4097, 4100), (70000, 70000)])
+def test_sample_equal_logits_are_bit_exact(V, stride):
+    # equal logits: every weight is 1 and every partial sum an integer, exact in fp32; with u a multiple of 2^-10
+    # u * V is exact too, so the token is floor(u * V) on both sides, boundaries included
+    rng = np.random.default_rng(V)
+    tb = H.make_trees([9, 30, 25], [3, 0, 8], rng, vocab=V)
+    N = tb.total_nodes
+    u = (rng.integers(0, 1024, N) / 1024.0).astype(np.float32)
+    u[:4] = [0.0, 0.5, 1023.0 / 1024.0, 0.25]
+    lg = np.full((N, stride), 1.25, dtype=np.float32)
+    lg[:, V:] = 99.0                                           # padding beyond the vocabulary is never read
+    g, path, n_path, nxt = H.run_accept(H.DevTrees(tb), lg, vocab=V, temperature=1.3, uniforms=u)
+    np.testing.assert_array_equal(g, oracle.sample_tokens(lg, 1.3, u, vocab=V))
+    np.testing.assert_array_equal(g, np.floor(u.astype(np.float64) * V).astype(np.int32))
+
+
+def test_sample_special_values_and_the_greedy_limit():
+    rng = np.random.default_rng(31)
+    tb = H.make_trees([12, 20], [4, 4], rng, vocab=9000)
+    N, V = tb.total_nodes, 9000
+    dt = H.DevTrees(tb)
+    u = rng.random(N).astype(np.float32)
+    one = np.full((N, V), -np.inf, dtype=np.float32)
+    pos = rng.integers(0, V, N)
+    one[np.arange(N), pos] = rng.standard_normal(N).astype(np.float32)
+    one[3, :] = np.nan                                         # nothing to draw from: 0
+    one[4, 8000] = np.inf                                      # a +inf logit takes everything
+    one[4, 8500] = np.inf
+    g = H.run_accept(dt, one, temperature=1.0, uniforms=u)[0]
+    exp = pos.copy()
+    exp[3] = 0
+    exp[4] = min(8000, pos[4]) if one[4, pos[4]] == np.inf else 8000
+    np.testing.assert_array_equal(g, exp)
+    np.testing.assert_array_equal(g, oracle.sample_tokens(one, 1.0, u))
+    lg = rng.standard_normal((N, V)).astype(np.float32)
+    lg[np.arange(N), pos] += 4.0                               # a clear maximum per row
+    lg[:, ::97] = np.nan                                       # NaN entries have no weight
+    lg[np.arange(N), pos] = np.where(np.isnan(lg[np.arange(N), pos]), 6.0, lg[np.arange(N), pos])
+    cold = H.run_accept(dt, lg, temperature=1e-3, uniforms=u)
+    greedy = H.run_accept(dt, lg)
+    for a, b in zip(cold, greedy):                             # temperature -> 0: the greedy call's results
+        np.testing.assert_array_equal(a, b)
+    g = H.run_accept(dt, lg, temperature=1.0, uniforms=u)[0]
+    assert not np.any(np.isnan(lg[np.arange(N), g]))
+    assert_valid_draws(lg, V, 1.0, u, g)
+
+
+def test_sample_rejects_bad_arguments():
+    rng = np.random.default_rng(5)
+    tb = H.make_trees([6], [2], rng, vocab=50)
+    dt = H.DevTrees(tb)
+    lg = torch.zeros((6, 50), dtype=torch.float32, device="cuda")
+    u = torch.zeros(6, dtype=torch.float32, device="cuda")
+    g = torch.zeros(6, dtype=torch.int32, device="cuda")
+    path = torch.zeros((1, 8), dtype=torch.int32, device="cuda")
+    n = torch.zeros(1, dtype=torch.int32, device="cuda")
+    nxt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    c = H.ctx()
+
+    def call(**kw):
+        return binding.accept_args(dt.desc(), 50, lg, 50, g, path, 8, n, nxt, **kw)
+    assert c.falcon_tree_accept(call(temperature=1.0, uniforms=u), check=False) == binding.OK
+    assert c.falcon_tree_accept(call(temperature=1.0), check=False) == binding.ERR_INVALID_ARG
+    assert c.falcon_tree_accept(call(temperature=-1.0, uniforms=u), check=False) == binding.ERR_INVALID_ARG
+    assert c.falcon_tree_accept(call(temperature=float("nan"), uniforms=u), check=False) == binding.ERR_INVALID_ARG
+    assert binding.falcon_tree_accept_static(call(temperature=1.0, uniforms=u), check=False) == binding.ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+
+
 # ------------------------------------------------------------------------ LM-head argmax (Section 3.1, Eq. 6)
 def assert_lm_argmax(f, w, hidden=None, tol=None):
     """The kernel sums in fp32 in the tensor core's order, the oracle in double: the maximum itself must agree
