@@ -19,6 +19,11 @@
 //     for the subsequent drafting phase" (Section 3.4), in its KV-cache form.
 //   * top-m selection (the step before verification): every tree node is expanded
 //     with the m most probable tokens of the drafter's distribution (Appendix A).
+//   * the LM head with the greedy token taken directly (Section 3.1, Eq. 6).
+//   * non-greedy decoding: the target's own draw at every node (Section 3.1).  The
+//     paper states no acceptance rule for this case; oracle_sample_tokens follows
+//     a reading stated at the function, so it is "parity unpinned" with respect to
+//     the paper (its arithmetic is pinned like the rest).
 //
 // Every routine is the plain definition: visible sets by walking parent
 // pointers, two-pass softmax with double accumulators, sequential argmax scan,
