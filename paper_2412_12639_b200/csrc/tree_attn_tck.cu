@@ -39,6 +39,8 @@
 // memory, and one prefix tile when the caller declared the prefix stable, come before
 // griddepcontrol.wait.  Every mbarrier wait is bounded; a wait that runs out sets FALCON_DEV_TIMEOUT,
 // what is in flight is drained, and the rows are still delivered (by the exact path).
+#include <algorithm>
+
 #include "tc_util.cuh"
 
 // Profiling hooks, empty by default: a private build may predefine them to record time stamps.
@@ -144,6 +146,8 @@ struct TckParams {
   int32_t prefetch_next;   // tm_nk / tm_nv describe the caches of the next call: bring their prefix tiles into L2
   int32_t h_node_off[kHostSeqs + 1];
   int32_t h_prefix[kHostSeqs];
+  int32_t h_order[kHostSeqs];  // grid z -> sequence, longest first (CTAs are handed out in grid order: with more
+                               // CTAs than SMs the long sequences must not be the ones that start last)
   FALCON_TRACE_PARAMS
 };
 
@@ -339,7 +343,8 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n_splits = gridDim.x, split = blockIdx.x;  // cluster = all CTAs of a row of the grid
-  const int kvh = blockIdx.y % p.Hkv, mtile = blockIdx.y / p.Hkv, b = blockIdx.z;
+  const int kvh = blockIdx.y % p.Hkv, mtile = blockIdx.y / p.Hkv;
+  const int b = p.have_host ? p.h_order[blockIdx.z] : static_cast<int>(blockIdx.z);
   constexpr int kCW = VT::kCW, kPer = VT::kPer;
   const int G = p.G, N = p.n_rows, n_chunks = N / kCW;
   const uint32_t q_half_bytes = static_cast<uint32_t>(N) * 128u;  // between the two 64-column halves of Q
@@ -1045,6 +1050,10 @@ int launch_impl(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream_t s, int 
     p.have_host = 1;
     for (int i = 0; i <= B; ++i) p.h_node_off[i] = a.tree.node_off_host[i];
     for (int i = 0; i < B; ++i) p.h_prefix[i] = a.tree.prefix_len_host[i];
+    for (int i = 0; i < B; ++i) p.h_order[i] = i;
+    std::stable_sort(p.h_order, p.h_order + B, [&](int x, int y) {
+      return p.h_prefix[x] + (p.h_node_off[x + 1] - p.h_node_off[x]) > p.h_prefix[y] + (p.h_node_off[y + 1] - p.h_node_off[y]);
+    });
   }
 
   FALCON_TRACE_LAUNCH(p)
