@@ -587,7 +587,8 @@ def test_attn_tc_random_batches_and_splits(seed, tck):
 # ----------------------------------------------------------------------- top-m
 @pytest.mark.parametrize("N,V,stride,m", [(1, 1, 1, 1), (3, 7, 9, 7), (5, 1000, 1000, 20), (60, 32000, 32000, 20),
                                           (4, 32001, 32005, 32), (2, 4099, 4101, 1), (2, 262144, 262144, 20),
-                                          (130, 5000, 5000, 5)])
+                                          (130, 5000, 5000, 5), (3, 8192, 8192, 20), (70, 65536, 65536, 32),
+                                          (9, 40000, 40000, 31)])
 def test_topm_bit_exact(N, V, stride, m):
     rng = np.random.default_rng(V + m)
     x = rng.standard_normal((N, stride)).astype(np.float32)
@@ -688,6 +689,20 @@ def test_sample_equal_logits_are_bit_exact(V, stride):
     np.testing.assert_array_equal(g, np.floor(u.astype(np.float64) * V).astype(np.int32))
 
 
+def test_sample_edge_sizes_and_the_last_representable_uniform():
+    rng = np.random.default_rng(41)
+    for sizes, V in (([1], 1), ([1], 5), ([2, 1, 3], 4096), ([5], 4097), ([3], 12289)):
+        tb = H.make_trees(sizes, [0] * len(sizes), rng, vocab=V)
+        N = tb.total_nodes
+        lg = rng.standard_normal((N, V)).astype(np.float32)
+        u = rng.random(N).astype(np.float32)
+        u[0] = np.float32(1.0) - np.float32(2.0 ** -24)        # the largest float below 1: the end of the row
+        if N > 1:
+            u[1] = 0.0                                         # the first token that has weight
+        g = H.run_accept(H.DevTrees(tb), lg, temperature=0.9, uniforms=u)[0]
+        assert_valid_draws(lg, V, 0.9, u, g)
+
+
 def test_sample_special_values_and_the_greedy_limit():
     rng = np.random.default_rng(31)
     tb = H.make_trees([12, 20], [4, 4], rng, vocab=9000)
@@ -762,7 +777,8 @@ def assert_lm_argmax(f, w, hidden=None, tol=None):
     return g, g_ref
 
 
-@pytest.mark.parametrize("N,Hd,V", [(60, 256, 1000), (7, 64, 40), (130, 192, 3001), (300, 128, 2500), (60, 128, 50000)])
+@pytest.mark.parametrize("N,Hd,V", [(60, 256, 1000), (7, 64, 40), (130, 192, 3001), (300, 128, 2500), (60, 128, 50000),
+                                    (1, 8, 1), (129, 64, 17), (2, 72, 2368), (64, 136, 2369)])
 def test_lm_head_argmax_integer_data_is_bit_exact(N, Hd, V):
     # small integers: every product and every partial sum is exact in fp32, so values, ties and indices must
     # equal the oracle's bit for bit (one node tile, two resident tiles, three tiles in two rounds; a vocabulary
@@ -770,8 +786,9 @@ def test_lm_head_argmax_integer_data_is_bit_exact(N, Hd, V):
     rng = np.random.default_rng(N + V)
     fi = rng.integers(-3, 4, size=(N, Hd))
     wi = rng.integers(-3, 4, size=(V, Hd))
-    wi[V // 2] = wi[5]                                         # identical head rows: a tie for every node
-    wi[V - 1] = wi[5]
+    if V > 8:
+        wi[V // 2] = wi[5]                                     # identical head rows: a tie for every node
+        wi[V - 1] = wi[5]
     f = synth.f32_to_bf16_bits(fi.astype(np.float32))
     w = synth.f32_to_bf16_bits(wi.astype(np.float32))
     g_ref, best_ref = oracle.lm_head_argmax(f, w)
