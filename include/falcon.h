@@ -243,6 +243,10 @@ int falcon_tree_accept(falcon_ctx* ctx, const falcon_accept_args* args, void* st
  *            wait inside the kernel gave up (the results are then not valid)
  * Device pointers; the caller owns every buffer; scratch comes from the context.
  * ------------------------------------------------------------------------- */
+/* Test hook: the features of the first pipeline stage are never requested, so the kernel's first
+ * bounded wait runs out: FALCON_DEV_TIMEOUT in *status, the kernel returns in order, the context
+ * stays usable.  (No fault, no hang: every wait in the kernel has a limit.) */
+#define FALCON_LM_TEST_STALL (1 << 30)
 typedef struct {
   int32_t n_rows;         /* N: rows of `features` (tree nodes)                        */
   int32_t hidden;
@@ -254,6 +258,7 @@ typedef struct {
   int32_t* argmax_out;    /* [n_rows]                                                  */
   float* max_out;         /* [n_rows] or NULL                                          */
   int32_t* status;        /* 1 word or NULL                                            */
+  int32_t flags;          /* 0, or FALCON_LM_TEST_STALL                                */
 } falcon_lm_argmax_args;
 
 int falcon_lm_head_argmax(falcon_ctx* ctx, const falcon_lm_argmax_args* args, void* stream);

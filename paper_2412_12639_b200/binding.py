@@ -60,7 +60,7 @@ class TopmArgs(C.Structure):
 class LmArgmaxArgs(C.Structure):
     _fields_ = [("n_rows", C.c_int32), ("hidden", C.c_int32), ("vocab", C.c_int32), ("features", C.c_void_p),
                 ("feat_stride", C.c_int64), ("lm_head", C.c_void_p), ("head_stride", C.c_int64),
-                ("argmax_out", C.c_void_p), ("max_out", C.c_void_p), ("status", C.c_void_p)]
+                ("argmax_out", C.c_void_p), ("max_out", C.c_void_p), ("status", C.c_void_p), ("flags", C.c_int32)]
 
 
 class GatherArgs(C.Structure):
@@ -127,6 +127,7 @@ def falcon_tree_validate_host(parent) -> int:
 
 STATIC_MAX_NODES, STATIC_MAX_BATCH = 1024, 256
 TOPM_MAX = 32
+LM_TEST_STALL = 1 << 30
 
 
 def falcon_tree_accept_static(args: "AcceptArgs", stream=None, check: bool = True) -> int:
@@ -255,9 +256,9 @@ def topm_args(n_rows, vocab, logits, logits_stride, m, top_val, top_idx) -> Topm
 
 
 def lm_argmax_args(n_rows, hidden, vocab, features, feat_stride, lm_head, head_stride, argmax_out, max_out=None,
-                   status=None) -> LmArgmaxArgs:
+                   status=None, flags=0) -> LmArgmaxArgs:
     return LmArgmaxArgs(n_rows, hidden, vocab, _ptr(features), feat_stride, _ptr(lm_head), head_stride,
-                        _ptr(argmax_out), _ptr(max_out), _ptr(status))
+                        _ptr(argmax_out), _ptr(max_out), _ptr(status), flags)
 
 
 def gather_args(tree: TreeDesc, hidden, features, feat_stride, path, path_stride, n_path, out_rows, features_out,

@@ -214,6 +214,7 @@ int falcon_lm_head_argmax(falcon_ctx* ctx, const falcon_lm_argmax_args* a, void*
   if ((a->feat_stride | a->head_stride) & 7) return FALCON_ERR_UNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(a->features) | reinterpret_cast<uintptr_t>(a->lm_head)) & 15) return FALCON_ERR_UNSUPPORTED;
   if (a->n_rows > 65535) return FALCON_ERR_CAPACITY;
+  if (a->flags & ~FALCON_LM_TEST_STALL) return FALCON_ERR_INVALID_ARG;
   return launch_lm_head_argmax(ctx, *a, static_cast<cudaStream_t>(stream));
 }
 

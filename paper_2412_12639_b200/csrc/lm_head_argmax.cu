@@ -58,6 +58,7 @@ struct LmParams {
   int32_t tile_n;     // vocabulary rows per MMA (multiple of 16)
   int32_t span;       // vocabulary rows per CTA (multiple of 16)
   int32_t n_stages;
+  int32_t stall_first;  // test hook: the features of ring stage 0 are never requested (a bounded wait then runs out)
   uint32_t stage_bytes, idesc;
   int32_t* argmax_out;
   float* max_out;
@@ -124,6 +125,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
       tma_load_5d(dst + c * w_bytes, &tm_w, bar(kLmBarFull + st), (kq * p.kch + c) * kLmKC, v_lo + vt * p.tile_n, 0, 0, 0);
   };
   auto issue_feat = [&](int it) {
+    if (it == 0 && p.stall_first) return;
     const int st = it % S, kq = (it % n_ks + rot) % n_ks, g = it / (n_ks * n_vt);
     const uint32_t fdst = smem_base + static_cast<uint32_t>(st) * p.stage_bytes + static_cast<uint32_t>(p.kch) * w_bytes;
     for (int c = 0; c < p.kch; ++c)
@@ -363,6 +365,7 @@ int launch_lm_head_argmax(falcon_ctx* ctx, const falcon_lm_argmax_args& a, cudaS
   p.tile_n = tile_n;
   p.span = span;
   p.n_stages = n_stages;
+  p.stall_first = (a.flags & FALCON_LM_TEST_STALL) ? 1 : 0;
   p.stage_bytes = stage_bytes;
   p.idesc = make_idesc(128, static_cast<uint32_t>(tile_n), false, false);
   p.argmax_out = a.argmax_out;

@@ -872,6 +872,30 @@ def test_lm_head_argmax_then_accept_from_the_argmax():
     np.testing.assert_array_equal(nxt.cpu().numpy(), rt)
 
 
+def test_lm_head_argmax_bounded_wait_runs_out_and_the_context_stays_usable():
+    # the test hook withholds the first stage's features: the MMA warp's wait gives up after its limit, every role
+    # leaves in order, the status word says so, and the next call on the same context is right
+    rng = np.random.default_rng(12)
+    N, Hd, V = 40, 256, 3000
+    fi = rng.integers(-3, 4, size=(N, Hd))
+    wi = rng.integers(-3, 4, size=(V, Hd))
+    f = synth.f32_to_bf16_bits(fi.astype(np.float32))
+    w = synth.f32_to_bf16_bits(wi.astype(np.float32))
+    fd, wd = H.dev_bf16(f), H.dev_bf16(w)
+    g = torch.zeros(N, dtype=torch.int32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    c = H.ctx()
+    rc = c.falcon_lm_head_argmax(binding.lm_argmax_args(N, Hd, V, fd, Hd, wd, Hd, g, None, st,
+                                                        flags=binding.LM_TEST_STALL), check=False)
+    torch.cuda.synchronize()
+    assert rc == 0 and int(st.item()) & binding.DEV_TIMEOUT
+    st.zero_()
+    c.falcon_lm_head_argmax(binding.lm_argmax_args(N, Hd, V, fd, Hd, wd, Hd, g, None, st))
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    np.testing.assert_array_equal(g.cpu().numpy(), oracle.lm_head_argmax(f, w)[0])
+
+
 def test_lm_head_argmax_rejects_bad_arguments_without_launching():
     f = torch.zeros((4, 72), dtype=torch.bfloat16, device="cuda")
     w = torch.zeros((10, 72), dtype=torch.bfloat16, device="cuda")
