@@ -19,6 +19,7 @@ namespace {
 
 constexpr int kWarpsPerCta = 4;
 constexpr int kWarpKeysMax = 1024;  // keys per sequence this kernel takes (scores live in shared memory)
+constexpr int kWarpHostSeqs = 8;    // sequences whose scalars travel in the kernel's parameters
 
 struct WarpParams {
   int32_t batch, Hq, Hkv, s_cap;
@@ -35,6 +36,9 @@ struct WarpParams {
   const __nv_bfloat16* k_tree;
   const __nv_bfloat16* v_tree;
   const uint64_t* tree_mask;
+  int32_t have_host;  // the caller's host copies of the per-sequence scalars came with the call
+  int32_t h_node_off[kWarpHostSeqs + 1];
+  int32_t h_prefix[kWarpHostSeqs];
 };
 
 __device__ __forceinline__ float ex2f(float x) {
@@ -51,41 +55,33 @@ __global__ void __launch_bounds__(32 * kWarpsPerCta) tree_attn_warp_kernel(const
   __shared__ float s_s[kWarpKeysMax];
   __shared__ float red_s[2][kWarpsPerCta];
   __shared__ float acc_s[kWarpsPerCta][D];
+  __shared__ int32_t par_s[FALCON_T_MAX];
 
   // Under programmatic dependent launch the grid may start while the previous kernel of the stream
   // drains: nothing is read or written before that kernel has completed.
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h = blockIdx.x, node = blockIdx.y, b = blockIdx.z;
-  const int base = p.node_off[b];
-  const int T_real = p.node_off[b + 1] - base;
+  // With the caller's host copies of the per-sequence scalars nothing has to be fetched before the
+  // addresses are known, and the query row, the tree's parent array and every thread's first key are
+  // asked for together: one round trip instead of a chain (scalars, then parents one by one, then keys).
+  int base, T_real, L_raw;
+  if (p.have_host) {
+    base = p.h_node_off[b];
+    T_real = p.h_node_off[b + 1] - base;
+    L_raw = p.h_prefix[b];
+  } else {
+    base = p.node_off[b];
+    T_real = p.node_off[b + 1] - base;
+    L_raw = p.prefix_len[b];
+  }
   const int T = min(T_real, FALCON_T_MAX);
   if (node >= T) return;  // the whole block
-  const int L = max(p.prefix_len[b], 0);
+  const int L = max(L_raw, 0);
   const bool separate = (p.k_tree != nullptr);
   const int prefix_rows = min(L, p.s_cap);
   const int S = min(separate ? prefix_rows + T : min(L + T, p.s_cap), kWarpKeysMax);
   const int G = p.Hq / p.Hkv, kvh = h / G;
-
-  // the query row first (its load overlaps the walk up the tree below)
-  const __nv_bfloat16* qrow = p.q + (static_cast<int64_t>(base + node) * p.Hq + h) * D;
-  if (tid < D) q_s[tid] = __bfloat162float(qrow[tid]);
-
-  uint64_t lo, hi;
-  bool bad = false;
-  if (p.tree_mask) {
-    lo = p.tree_mask[2 * static_cast<int64_t>(base + node)];
-    hi = p.tree_mask[2 * static_cast<int64_t>(base + node) + 1];
-  } else {
-    bad = !ancestor_mask(p.parent + base, T, node, lo, hi);
-    if (node == 0 && p.parent[base] != -1) bad = true;
-  }
-  if (tid == 0 && h == 0) {
-    if (bad) dev_status_or(p.status, b, FALCON_DEV_BAD_TREE);
-    if (node == 0 && (L + (separate ? 0 : T) > p.s_cap || T_real > FALCON_T_MAX || L + T > kWarpKeysMax))
-      dev_status_or(p.status, b, FALCON_DEV_CAPACITY);
-  }
-  __syncthreads();
 
   const __nv_bfloat16* kb = p.k_cache + b * p.stride_b + kvh * p.stride_h;
   const __nv_bfloat16* vb = p.v_cache + b * p.stride_b + kvh * p.stride_h;
@@ -95,33 +91,71 @@ __global__ void __launch_bounds__(32 * kWarpsPerCta) tree_attn_warp_kernel(const
     return cache + static_cast<int64_t>(key) * p.stride_s;
   };
 
+  const __nv_bfloat16* qrow = p.q + (static_cast<int64_t>(base + node) * p.Hq + h) * D;
+  __nv_bfloat16 q_raw = __float2bfloat16(0.f);
+  if (tid < D) q_raw = qrow[tid];
+  int par_raw = -1;
+  if (!p.tree_mask && tid < T) par_raw = p.parent[base + tid];
+  uint4 kx0[D / 8];
+  if (tid < S) {  // (masked or not: which tree keys count is known only after the walk below)
+    const uint4* kr = reinterpret_cast<const uint4*>(row_of(kb, p.k_tree, tid));
+#pragma unroll
+    for (int c = 0; c < D / 8; ++c) kx0[c] = kr[c];
+  }
+  if (tid < D) q_s[tid] = __bfloat162float(q_raw);
+  if (tid < T) par_s[tid] = par_raw;
+  __syncthreads();
+
+  uint64_t lo, hi;
+  bool bad = false;
+  if (p.tree_mask) {
+    lo = p.tree_mask[2 * static_cast<int64_t>(base + node)];
+    hi = p.tree_mask[2 * static_cast<int64_t>(base + node) + 1];
+  } else {
+    bad = !ancestor_mask(par_s, T, node, lo, hi);  // the walk, in shared memory
+    if (node == 0 && par_s[0] != -1) bad = true;
+  }
+  if (tid == 0 && h == 0) {
+    if (bad) dev_status_or(p.status, b, FALCON_DEV_BAD_TREE);
+    if (node == 0 && (L + (separate ? 0 : T) > p.s_cap || T_real > FALCON_T_MAX || L + T > kWarpKeysMax))
+      dev_status_or(p.status, b, FALCON_DEV_CAPACITY);
+  }
+
   // ---- pass 1: scores (one key per thread and round), row maximum ----
+  auto score = [&](const uint4 (&kx)[D / 8]) -> float {
+    float acc = 0.f;
+#pragma unroll
+    for (int c = 0; c < D / 8; ++c) {
+      const float4 qa = *reinterpret_cast<const float4*>(&q_s[8 * c]);
+      const float4 qb = *reinterpret_cast<const float4*>(&q_s[8 * c + 4]);
+      const __nv_bfloat162* kh = reinterpret_cast<const __nv_bfloat162*>(&kx[c]);
+      const float2 k0 = __bfloat1622float2(kh[0]), k1 = __bfloat1622float2(kh[1]);
+      const float2 k2 = __bfloat1622float2(kh[2]), k3 = __bfloat1622float2(kh[3]);
+      acc = fmaf(qa.x, k0.x, acc);
+      acc = fmaf(qa.y, k0.y, acc);
+      acc = fmaf(qa.z, k1.x, acc);
+      acc = fmaf(qa.w, k1.y, acc);
+      acc = fmaf(qb.x, k2.x, acc);
+      acc = fmaf(qb.y, k2.y, acc);
+      acc = fmaf(qb.z, k3.x, acc);
+      acc = fmaf(qb.w, k3.y, acc);
+    }
+    return acc * p.scale_log2;
+  };
   float mx = -INFINITY;
-  for (int key = tid; key < S; key += kThreads) {
+  if (tid < S) {  // this thread's first key is in registers already
+    const float s = (tid < prefix_rows || bit128(lo, hi, tid - prefix_rows)) ? score(kx0) : -INFINITY;
+    s_s[tid] = s;
+    mx = s;
+  }
+  for (int key = tid + kThreads; key < S; key += kThreads) {
     float s = -INFINITY;
     if (key < prefix_rows || bit128(lo, hi, key - prefix_rows)) {
       const uint4* kr = reinterpret_cast<const uint4*>(row_of(kb, p.k_tree, key));
       uint4 kx[D / 8];
 #pragma unroll
       for (int c = 0; c < D / 8; ++c) kx[c] = kr[c];
-      float acc = 0.f;
-#pragma unroll
-      for (int c = 0; c < D / 8; ++c) {
-        const float4 qa = *reinterpret_cast<const float4*>(&q_s[8 * c]);
-        const float4 qb = *reinterpret_cast<const float4*>(&q_s[8 * c + 4]);
-        const __nv_bfloat162* kh = reinterpret_cast<const __nv_bfloat162*>(&kx[c]);
-        const float2 k0 = __bfloat1622float2(kh[0]), k1 = __bfloat1622float2(kh[1]);
-        const float2 k2 = __bfloat1622float2(kh[2]), k3 = __bfloat1622float2(kh[3]);
-        acc = fmaf(qa.x, k0.x, acc);
-        acc = fmaf(qa.y, k0.y, acc);
-        acc = fmaf(qa.z, k1.x, acc);
-        acc = fmaf(qa.w, k1.y, acc);
-        acc = fmaf(qb.x, k2.x, acc);
-        acc = fmaf(qb.y, k2.y, acc);
-        acc = fmaf(qb.z, k3.x, acc);
-        acc = fmaf(qb.w, k3.y, acc);
-      }
-      s = acc * p.scale_log2;
+      s = score(kx);
     }
     s_s[key] = s;
     mx = fmaxf(mx, s);
@@ -220,6 +254,12 @@ int launch_tree_attn_warp(falcon_ctx* ctx, const falcon_attn_args& a, cudaStream
   p.k_tree = static_cast<const __nv_bfloat16*>(a.k_tree);
   p.v_tree = static_cast<const __nv_bfloat16*>(a.v_tree);
   p.tree_mask = a.tree_mask;
+  p.have_host = 0;
+  if (a.tree.prefix_len_host && a.tree.node_off_host && a.tree.batch <= kWarpHostSeqs) {
+    p.have_host = 1;
+    for (int i = 0; i <= a.tree.batch; ++i) p.h_node_off[i] = a.tree.node_off_host[i];
+    for (int i = 0; i < a.tree.batch; ++i) p.h_prefix[i] = a.tree.prefix_len_host[i];
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(a.n_q_heads, a.tree.max_tree, a.tree.batch);
   cfg.blockDim = dim3(32 * kWarpsPerCta);
