@@ -48,14 +48,16 @@ def accept_bytes(spec, tb) -> int:
     return 4 * tb.total_nodes * spec.vocab + 12 * tb.total_nodes
 
 
-def recorded_traffic(workload: str, kernel: str):
-    """DRAM bytes per attention launch from the committed ncu summary of this workload and kernel ("tc", "tck"),
-    or None when there is none or the kernel source has changed since the counters were taken."""
+def recorded_traffic(workload: str, kernel: str, stem: str = "tree_attn_%s"):
+    """DRAM bytes per launch from the committed ncu summary of this workload and kernel (attention: "tc", "tck";
+    stem "lm_head_argmax" for that kernel), or None when there is none or the kernel source has changed since
+    the counters were taken."""
     import hashlib
     import re
+    name = stem % kernel if "%s" in stem else stem
     try:
-        text = open(os.path.join(ROOT, "profiles", "tree_attn_%s_%s_ncu.md" % (kernel, workload))).read()
-        src = open(os.path.join(ROOT, "paper_2412_12639_b200", "csrc", "tree_attn_%s.cu" % kernel), "rb").read()
+        text = open(os.path.join(ROOT, "profiles", "%s_%s_ncu.md" % (name, workload))).read()
+        src = open(os.path.join(ROOT, "paper_2412_12639_b200", "csrc", "%s.cu" % name), "rb").read()
     except OSError:
         return None
     sha = re.search(r"kernel_source_sha256:\s*([0-9a-f]{64})", text)
@@ -254,7 +256,7 @@ def time_topm(ctx, binding, torch, dev, stream, logits_h, peak, m=20, copies=20,
                          "traffic": None}}
 
 
-def time_lm_head(ctx, binding, torch, dev, stream, n_rows, hidden, vocab, peak, reps=10):
+def time_lm_head(ctx, binding, torch, dev, stream, n_rows, hidden, vocab, peak, workload, reps=10):
     """falcon_lm_head_argmax (Section 3.1, Eq. 6: the LM head applied to the nodes' features, greedy token only)
     at the workload's shape, hidden = query heads x head_dim: two distinct random heads alternate (together more
     than L2) in one CUDA graph, replayed; CUDA events on the launching stream.  Not part of the step."""
@@ -288,7 +290,7 @@ def time_lm_head(ctx, binding, torch, dev, stream, n_rows, hidden, vocab, peak, 
     return {"rows": n_rows, "hidden": hidden, "vocab": vocab, "us_per_call": us, "bytes_per_call": nbytes,
             "useful_tflops": 2.0 * n_rows * hidden * vocab / (us * 1e-6) / 1e12,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                         "traffic": None}}
+                         "traffic": recorded_traffic(workload, "", stem="lm_head_argmax")}}
 
 
 # --------------------------------------------------------------------------- GPU arm
@@ -482,8 +484,8 @@ def run_falcon(args):
 
     # ---------------- outside the step: the selection that grows the tree (the row next to the hot path) ----
     topm = time_topm(ctx, binding, torch, dev, stream, logits_h, peak) if world == 1 else None
-    lm = (time_lm_head(ctx, binding, torch, dev, stream, tb.total_nodes, spec.n_q_heads * spec.head_dim, spec.vocab, peak)
-          if world == 1 else None)
+    lm = (time_lm_head(ctx, binding, torch, dev, stream, tb.total_nodes, spec.n_q_heads * spec.head_dim, spec.vocab, peak,
+                       args.workload) if world == 1 else None)
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
