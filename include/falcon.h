@@ -185,8 +185,8 @@ int falcon_tree_attn_kernel(falcon_ctx* ctx, const falcon_attn_args* args);
  *   n_path[b] = nodes on the path (accepted drafted tokens = n_path - 1)
  *   next_token[b] = g[last node of the path]
  *
- * Non-greedy decoding (temperature > 0).  Section 3.1: the LM head gives the
- * probability distribution "from which the next token is sampled"; the paper
+ * Non-greedy decoding (temperature > 0).  Section 3.1: the next token is drawn
+ * from the distribution that the LM head computes; the paper
  * states no acceptance rule for this case (Appendix A only says the drafted
  * children are sampled; Section 3.4 that verification follows SpecInfer).  The
  * rule here is the simplest one that leaves the output distribution the target's
@@ -220,8 +220,8 @@ int falcon_tree_accept(falcon_ctx* ctx, const falcon_accept_args* args, void* st
 
 /* ---------------------------------------------------------------------------
  * falcon_lm_head_argmax - the greedy token of every tree node straight from the
- * LM head (Section 3.1: "the LM Head computes the probability distribution based
- * on the aggregated features"; Eq. 6: p = Softmax(LM(f)); at temperature 0,
+ * LM head (Section 3.1: the LM head turns the aggregated features into the
+ * distribution over the vocabulary; Eq. 6: p = Softmax(LM(f)); at temperature 0,
  * Section 4.1, only the position of the largest logit matters).  The [N, vocab]
  * logits are never written to memory:
  *
@@ -265,8 +265,8 @@ int falcon_lm_head_argmax(falcon_ctx* ctx, const falcon_lm_argmax_args* args, vo
 
 /* ---------------------------------------------------------------------------
  * falcon_topm - the m best entries of every logits row, best first: the children
- * a node of the decoding tree is given when the tree is grown (Appendix A: "the m
- * tokens with the highest probability", m = 20 at the root).  It is the step just
+ * a node of the decoding tree is given when the tree is grown (Appendix A: in the
+ * greedy setting the m most probable tokens, m = 20 at the root).  It is the step just
  * before verification and scans the same kind of [rows, vocab] fp32 matrix as
  * the acceptance call.
  *
@@ -321,9 +321,8 @@ int falcon_tree_accept_static(const falcon_accept_args* args, void* stream);
 
 /* ---------------------------------------------------------------------------
  * falcon_feature_gather - the accepted tokens and their features (Section 3.4: after
- * verification "we record the accepted tokens and their corresponding features for the
- * subsequent drafting phase": the drafter's next input is the target model's hidden state
- * of every accepted node together with its token, Section 3.1).
+ * verification they are kept for the next drafting phase: the drafter's next input is the
+ * target model's hidden state of every accepted node together with its token, Section 3.1).
  *
  *   tokens_out[b, j]      = token[node_off[b] + path[b][j]]
  *   features_out[b, j, :] = features[node_off[b] + path[b][j], 0 .. hidden-1]    j < n_path[b]
@@ -351,9 +350,9 @@ typedef struct {
 int falcon_feature_gather(falcon_ctx* ctx, const falcon_gather_args* args, void* stream);
 
 /* ---------------------------------------------------------------------------
- * falcon_kv_compact - keep the accepted path's K/V (Section 3.4: "record the
- * accepted tokens and their corresponding features for the subsequent drafting
- * phase", in its KV-cache form), all layers in one launch.
+ * falcon_kv_compact - keep the accepted path's K/V (Section 3.4: the accepted tokens
+ * and their features are kept for the next drafting phase; this is the KV-cache form
+ * of that step), all layers in one launch.
  *
  *   cache row L_b + j  <-  tree row path[b][j],   j = 0 .. n_path[b]-1
  *   new_len[b] = L_b + n_path[b]

@@ -8,15 +8,15 @@
 // What is computed, and where the paper says so:
 //   * tree-masked attention: the target model scores all drafted tree tokens in
 //     one forward pass, each token attending to the sequence's prefix and to its
-//     own root-to-node chain ("tree-based parallel decoding ... consistent with
-//     SpecInfer", Section 3.4; "tree attention in both drafting and verification
-//     phases", Section 4.5).  The paper writes no attention formula; standard
+//     own root-to-node chain (Section 3.4 verifies the whole tree in one parallel
+//     pass the way SpecInfer does; Section 4.5 uses tree attention when drafting
+//     and when verifying).  The paper writes no attention formula; standard
 //     scaled-dot-product softmax is taken.
 //   * greedy acceptance: temperature 0 (Section 4.1); a drafted child is accepted
 //     when its token equals the target's argmax at its parent; the accepted
 //     length is the tau of Section 4.2.
-//   * compaction: "record the accepted tokens and their corresponding features
-//     for the subsequent drafting phase" (Section 3.4), in its KV-cache form.
+//   * compaction: after verification the accepted tokens and their features are
+//     kept for the next drafting phase (Section 3.4); this is the KV-cache form.
 //   * top-m selection (the step before verification): every tree node is expanded
 //     with the m most probable tokens of the drafter's distribution (Appendix A).
 //   * the LM head with the greedy token taken directly (Section 3.1, Eq. 6).
@@ -54,7 +54,7 @@ inline float bf16_to_float(uint16_t h) {
 }
 
 // A(i): node i, its parent, its grandparent, ... up to the root (Section 3.4:
-// a token sees "their predecessors in the tree"; verification uses the strict
+// a token sees the tokens that precede it in the tree; verification uses the strict
 // ancestor-or-self set).  Returns false on a malformed tree.
 bool ancestor_chain(const int32_t* parent, int32_t T, int32_t i, std::vector<int32_t>& chain) {
   chain.clear();
@@ -259,10 +259,10 @@ int oracle_argmax(const float* logits, int32_t N, int32_t V, int64_t stride, int
   return 0;
 }
 
-// The target model's own token at every node when decoding is not greedy.  Section 3.1: the LM
-// head gives "the probability distribution ..., from which the next token is sampled"; Appendix A
-// only says that in a non-greedy setting the drafted children are sampled, and Section 3.4 that
-// verification is "consistent with SpecInfer" - the paper states no acceptance rule of its own.
+// The target model's own token at every node when decoding is not greedy.  Section 3.1: the next
+// token is drawn from the distribution that the LM head computes; Appendix A only says that in a
+// non-greedy setting the drafted children are sampled, and Section 3.4 that verification follows
+// SpecInfer - the paper states no acceptance rule of its own.
 // The reading taken here is the simplest lossless one: at every node the target draws its token
 // from softmax(logits / temperature), and a drafted child is accepted when it carries that token
 // (with temperature -> 0 this is the greedy rule).  The draw is the inverse-CDF one, with the
@@ -318,8 +318,8 @@ int oracle_sample_tokens(const float* logits, int32_t N, int32_t V, int64_t stri
 }
 
 // LM-head logits of the tree's nodes and their greedy argmax without a logits matrix in
-// between.  The verification pass ends in the target model's LM head: "the LM Head computes
-// the probability distribution based on the aggregated features" (Section 3.1) and Eq. 6 writes
+// between.  The verification pass ends in the target model's LM head, which turns the
+// aggregated features into the distribution over the vocabulary (Section 3.1); Eq. 6 writes
 // p = Softmax(LM(f)); with temperature 0 (Section 4.1) only the position of the largest logit
 // is needed, and the softmax does not move it.  The LM head is taken as a bias-free linear map
 // (the LLaMA / Vicuna heads the paper evaluates have no bias):
@@ -356,7 +356,7 @@ int oracle_lm_head_argmax(const uint16_t* feat, int64_t feat_stride, const uint1
 }
 
 // Top-m entries of every row, best first: the children a tree node is given when the tree is
-// grown ("the m tokens with the highest probability", Appendix A; m = 20 at the root there).
+// grown (in the greedy setting the m most probable tokens, Appendix A; m = 20 at the root there).
 // Plain definition: m passes over the row, each taking the best entry not taken yet.  Order:
 // larger value first, the lower index among equal values (+0 and -0 are equal); a NaN counts as
 // -inf and is reported as -inf.  Needs 1 <= m <= V.
@@ -499,8 +499,8 @@ int oracle_kv_compact(int32_t B, const int32_t* node_off, const int32_t* prefix_
   return 0;
 }
 
-// Accepted tokens and their features (Section 3.4: "record the accepted tokens and their
-// corresponding features for the subsequent drafting phase"): for every node on the accepted
+// Accepted tokens and their features (Section 3.4: they are kept after verification, as the
+// input of the next drafting phase): for every node on the accepted
 // path, in path order, its drafted token and its row of the [N, hidden] feature matrix (16-bit
 // elements, copied bit for bit).  feat_out is [B, out_rows, hidden], tok_out [B, out_rows]; only
 // the first n_path[b] rows of a sequence are written.

@@ -41,7 +41,7 @@ struct CompactParams {
 };
 
 // Accepted tokens and features of sequence b: an out-of-place row gather along the path (Section
-// 3.4, "record the accepted tokens and their corresponding features").  The `n_parts` CTAs of a
+// 3.4: the accepted tokens and their features are kept for the next drafting phase).  The `n_parts` CTAs of a
 // sequence share the 16-byte chunks; the path has been validated into s_path by the caller.
 __device__ __forceinline__ void gather_features(const CompactParams& p, int b, int base, int n, const int* s_path,
                                                 int part, int n_parts, int tid) {

@@ -1,6 +1,6 @@
 // falcon_lm_head_argmax: the greedy token of every tree node straight from the LM head
-// (Section 3.1: "the LM Head computes the probability distribution based on the aggregated
-// features"; Eq. 6: p = Softmax(LM(f)); temperature 0, Section 4.1, needs only the position of the
+// (Section 3.1: the LM head turns the aggregated features into the distribution over the
+// vocabulary; Eq. 6: p = Softmax(LM(f)); temperature 0, Section 4.1, needs only the position of the
 // largest logit).  logit[i, v] = sum_k feat[i, k] * head[v, k] is a dense bf16 contraction whose
 // [N, V] fp32 result is never written: the argmax is taken where the accumulator is read.
 //
