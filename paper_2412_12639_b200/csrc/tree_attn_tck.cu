@@ -174,6 +174,19 @@ __device__ __forceinline__ void prefetch_tile_l2(const CUtensorMap* map, int key
                : "memory");
 }
 
+// (d0, d1) = (a0, a1) * (b0, b1) + (c0, c1) in one instruction
+__device__ __forceinline__ void fma2(float a0, float a1, float b0, float b1, float c0, float c1, float& d0, float& d1) {
+  asm("{ .reg .b64 ra, rb, rc, rd; mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %5}; mov.b64 rc, {%6, %7}; "
+      "fma.rn.f32x2 rd, ra, rb, rc; mov.b64 {%0, %1}, rd; }"
+      : "=f"(d0), "=f"(d1)
+      : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
+}
+// (x0, x1) += (y0, y1) in one instruction
+__device__ __forceinline__ void add2(float& x0, float& x1, float y0, float y1) {
+  asm("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%0, %1}; mov.b64 rb, {%2, %3}; add.rn.f32x2 rd, ra, rb; mov.b64 {%0, %1}, rd; }"
+      : "+f"(x0), "+f"(x1)
+      : "f"(y0), "f"(y1));
+}
 template <int kW>
 __device__ __forceinline__ void tmem_ld_chunk(uint32_t taddr, uint32_t (&r)[kW]) {
   if constexpr (kW == 16) {
@@ -765,8 +778,11 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
           uint32_t pk[kCW / 2];
 #pragma unroll
           for (int c = 0; c < kCW; c += 2) {
-            float p0 = ex2(fmaf(__uint_as_float(sr[cr][c]), scale, neg_ref[cr][c]));
-            float p1 = ex2(fmaf(__uint_as_float(sr[cr][c + 1]), scale, neg_ref[cr][c + 1]));
+            // two columns at a time: one packed fma for the exponents, one packed add for the row sums
+            float e0, e1;
+            fma2(__uint_as_float(sr[cr][c]), __uint_as_float(sr[cr][c + 1]), scale, scale, neg_ref[cr][c], neg_ref[cr][c + 1],
+                 e0, e1);
+            float p0 = ex2(e0), p1 = ex2(e1);
             if (!full) {
               p0 = ((vis >> c) & 1u) ? p0 : 0.f;
               p1 = ((vis >> (c + 1)) & 1u) ? p1 : 0.f;
@@ -776,8 +792,7 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             // that one key dominates is exact whatever that key's weight is).
             const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
             pk[c >> 1] = __byte_perm(b0, b1, 0x7632);
-            l_acc[ci][c] += __uint_as_float(b0 & 0xffff0000u);
-            l_acc[ci][c + 1] += __uint_as_float(b1 & 0xffff0000u);
+            add2(l_acc[ci][c], l_acc[ci][c + 1], __uint_as_float(b0 & 0xffff0000u), __uint_as_float(b1 & 0xffff0000u));
           }
           // P^T row of this key: the chunk's columns are 16-byte units (8 columns each) of the
           // 64-column block they fall in, swizzled by the row like everything the MMA reads
