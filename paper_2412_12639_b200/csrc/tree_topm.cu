@@ -13,7 +13,8 @@
 // order (key 0 = "no entry") only once they have survived.
 //   A  grid (chunks, rows), 8 warps per CTA: each warp loads its share of the CTA's chunk (up to
 //      16 or 32 entries per lane) straight into registers and leaves its survivors in shared memory;
-//   B  warp 0 thins the CTA's survivors again and writes them to scratch;
+//   B  the survivors go to scratch as they are (a second threshold over the whole CTA, from the
+//      warps' four largest lane maxima, keeps them to a few dozen), or thinned by warp 0 if more than 64;
 //   C  the last CTA of a row to finish (arrival counter) spreads the chunks' survivors over
 //      its 8 warps (eight chunks each);  D  its warp 0 thins the warps' survivors once more if more
 //      than one warp had any, ranks the at most 64 that remain and writes the first m.
@@ -40,6 +41,7 @@ static_assert(FALCON_TOPM_MAX <= kTopmCap, "the exact selection's m entries fit 
 struct TopmParams {
   int32_t n_rows, vocab, m, chunks, chunk_len;
   int32_t warp_span;   // entries of a chunk that one warp takes (a multiple of 32, at most 32 * kTopmRowsMax)
+  int32_t cta_thresh;  // pass A also uses a threshold over the whole CTA (see warp_thin_first)
   int64_t logits_stride;
   const float* logits;
   float* top_val;
@@ -138,7 +140,7 @@ __device__ __forceinline__ int warp_reserve(int* fill, int total, int lane) {
 // only the later passes, which work on keys, can tell whether it belongs).
 template <int kRows>
 __device__ __forceinline__ int warp_thin_first(const float* rowp, int n_w, int id0, int m, int lane, float* out_val, int* out_id,
-                                               int* fill) {
+                                               int* fill, uint32_t* cta_top, bool use_cta_top) {
   float x[kRows];
 #pragma unroll
   for (int k = 0; k < kRows; ++k) x[k] = (k * 32 + lane < n_w) ? rowp[k * 32 + lane] : -INFINITY;
@@ -148,7 +150,28 @@ __device__ __forceinline__ int warp_thin_first(const float* rowp, int n_w, int i
   float lm = x[0];
 #pragma unroll
   for (int k = 1; k < kRows; ++k) lm = fmaxf(lm, x[k]);
-  const float tau = from_key(warp_kth_largest(to_key(lm), m - 1, lane));
+  // The warp's threshold and, if asked for, a tighter one for the whole CTA (every warp of the CTA is here
+  // then): the four largest lane maxima of each of its 8 warps are 32 different entries, so their m-th
+  // largest is reached by at least m entries of the chunk.  With it the CTA's survivors are mostly few enough
+  // to go to the row as they are, without a pass of their own: fewer instructions, but a block-wide barrier in
+  // the middle of the pass.  The launcher asks for it when the grid is more than one wave (throughput counts);
+  // in a single wave the warps are better left to run ahead of one another (60 x 32000: 11.3 against 12.5 us).
+  const uint32_t lk = to_key(lm);
+  int rank = 0;
+#pragma unroll 4
+  for (int j = 0; j < 32; ++j) {
+    const uint32_t o = __shfl_sync(0xffffffffu, lk, j);
+    rank += (o > lk || (o == lk && j < lane)) ? 1 : 0;
+  }
+  if (rank < 4) cta_top[4 * (threadIdx.x >> 5) + rank] = lk;
+  const unsigned hit = __ballot_sync(0xffffffffu, rank == m - 1);
+  const uint32_t tau_w = __shfl_sync(0xffffffffu, lk, __ffs(static_cast<int>(hit)) - 1);
+  uint32_t tau_c = 0u;
+  if (use_cta_top) {
+    __syncthreads();
+    tau_c = warp_kth_largest(cta_top[lane], m - 1, lane);
+  }
+  const float tau = from_key(max(tau_w, tau_c));
   uint32_t mask = 0u;
 #pragma unroll
   for (int k = 0; k < kRows; ++k)
@@ -223,6 +246,7 @@ __global__ void __launch_bounds__(kTopmThreads, kRows <= 16 ? 4 : 3) tree_topm_k
   __shared__ int s_id[kTopmWarps * kTopmCap];
   __shared__ uint32_t s_fin_key[kTopmCap];
   __shared__ int s_fin_id[kTopmCap];
+  __shared__ uint32_t s_top[4 * kTopmWarps];  // the four largest lane maxima of every warp (pass A)
   __shared__ int s_fill;
   __shared__ int s_last;
 
@@ -242,7 +266,7 @@ __global__ void __launch_bounds__(kTopmThreads, kRows <= 16 ? 4 : 3) tree_topm_k
   {
     const int w0 = warp * p.warp_span;
     const int n_w = max(0, min(p.warp_span, n - w0));
-    warp_thin_first<kRows>(rowp + w0, n_w, c0 + w0, m, lane, reinterpret_cast<float*>(s_key), s_id, &s_fill);
+    warp_thin_first<kRows>(rowp + w0, n_w, c0 + w0, m, lane, reinterpret_cast<float*>(s_key), s_id, &s_fill, s_top, p.cta_thresh != 0);
   }
   __syncthreads();
 
@@ -259,12 +283,25 @@ __global__ void __launch_bounds__(kTopmThreads, kRows <= 16 ? 4 : 3) tree_topm_k
     }
   };
 
-  // ---- B: warp 0 thins the CTA's survivors and hands them to the row ----
-  if (warp == 0) {
+  // ---- B: the CTA's survivors go to the row: as they are when they are few enough, else thinned by warp 0 ----
+  const int64_t po = static_cast<int64_t>(row) * p.chunks + chunk;
+  const int fill_a = s_fill;
+  if (fill_a <= kTopmCap) {
+    if (tid < fill_a) {
+      p.part_key[po * kTopmCap + tid] = to_key(__uint_as_float(s_key[tid]));
+      p.part_idx[po * kTopmCap + tid] = s_id[tid];
+    }
+    __syncthreads();  // every thread's entries before thread 0's fence
+    if (tid == 0) {
+      p.part_cnt[po] = fill_a;
+      s_fill = 0;
+      __threadfence();
+      s_last = (atomicAdd(&p.tickets[row], 1) == p.chunks - 1);
+    }
+  } else if (warp == 0) {
     uint32_t key[kTopmPerLane];
     int id[kTopmPerLane];
     from_list(key, id, true);
-    const int64_t po = static_cast<int64_t>(row) * p.chunks + chunk;
     const int cnt = warp_thin(key, id, m, lane, p.part_key + po * kTopmCap, p.part_idx + po * kTopmCap, nullptr);
     __syncwarp();  // every lane's entries before lane 0's fence
     if (lane == 0) {
@@ -373,6 +410,8 @@ int launch_tree_topm(falcon_ctx* ctx, const falcon_topm_args& a, cudaStream_t s)
   p.chunks = chunks;
   p.chunk_len = chunk_len;
   p.warp_span = warp_span;
+  // (CTAs resident per SM: 4 with 16 entries per lane, 3 with 32: the kernel's launch bounds)
+  p.cta_thresh = static_cast<int64_t>(N) * chunks > static_cast<int64_t>(warp_span <= 16 * 32 ? 4 : 3) * ctx->sm_count ? 1 : 0;
   p.logits_stride = a.logits_stride;
   p.logits = a.logits;
   p.top_val = a.top_val;
