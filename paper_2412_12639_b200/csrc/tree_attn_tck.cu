@@ -110,7 +110,8 @@ struct Cfg {
   static constexpr uint32_t kDescWords = kN / 32;
   static constexpr uint32_t kOffDesc = 0;                                // [128 tree keys][kN / 32] words
   static constexpr uint32_t kOffRef = kOffDesc + 128 * kDescWords * 4;   // [kN] fp32
-  static constexpr uint32_t kOffRescue = kOffRef + kN * 4;               // [kN] bytes
+  static constexpr uint32_t kOffLpart = kOffRef + kN * 4;                // [4][kN] fp32: the lane quadrants' shares of the row sums
+  static constexpr uint32_t kOffRescue = kOffLpart + 16 * kN;            // [kN] bytes
   static constexpr uint32_t kOffPar = kOffRescue + kN;                   // [128] int8: the tree's parent array
   static constexpr uint32_t kOffBars = kOffPar + 128;
   static constexpr uint32_t kOffMisc = kOffBars + 8 * kNumBars;          // tmem base, abort flag
@@ -823,14 +824,42 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                                             : smem_base + off_mrg + static_cast<uint32_t>(split < owner ? split : split - 1) * slot_bytes;
       return map_to_rank(local, static_cast<uint32_t>(owner));
     };
-    bool have = live && n_my > 0 && !*abort_flag;
-    if (have) have = mbar_wait_warp(bar(kBarODone), 0, abort_flag);
+    const bool have = live && n_my > 0 && !*abort_flag;
+    if (n_splits > 1) cluster_wait();  // phase 1 (arrived long ago): every peer's merge barrier is initialised
+    // The row sums first: they are complete with the last tile's softmax pass and do not have to wait for the
+    // MMAs that are still running (Q is free by now: the last scores could only come after every QK product,
+    // so this split's own slot, which lies over Q, may be written).
+    float* s_lpart = reinterpret_cast<float*>(small + C::kOffLpart);
+#pragma unroll
+    for (int ci = 0; ci < kPer; ++ci) {
+      const int ch = grp + kColGroups * ci;
+      if (ch < n_chunks) {
+        // this warp's 32 keys' share of the chunk's row sums
+        const float sum = warp_col_sums<kCW>(l_acc[ci], lane);
+        if ((lane & (kCW == 16 ? 1 : 17)) == 0) s_lpart[q4 * C::kN + ch * kCW + col_of_lane<kCW>(lane)] = have ? sum : 0.f;
+      }
+    }
+    // the four lane quadrants' shares added (fixed order), four rows per thread, to every CTA (fp32, 4 bytes a
+    // query row, in the space of two more rows of the slot)
+    asm volatile("bar.sync 1, %0;" ::"n"(kSmThreads) : "memory");
+    if (st_id * 4 < N) {
+      const float4 s0 = reinterpret_cast<const float4*>(s_lpart)[st_id];
+      const float4 s1 = reinterpret_cast<const float4*>(s_lpart + C::kN)[st_id];
+      const float4 s2 = reinterpret_cast<const float4*>(s_lpart + 2 * C::kN)[st_id];
+      const float4 s3 = reinterpret_cast<const float4*>(s_lpart + 3 * C::kN)[st_id];
+      const uint32_t l0 = __float_as_uint((s0.x + s1.x) + (s2.x + s3.x)), l1 = __float_as_uint((s0.y + s1.y) + (s2.y + s3.y));
+      const uint32_t l2 = __float_as_uint((s0.z + s1.z) + (s2.z + s3.z)), l3 = __float_as_uint((s0.w + s1.w) + (s2.w + s3.w));
+      for (int i = 0; i < n_splits; ++i)
+        st_async_v4(slot_addr(i) + static_cast<uint32_t>(d_per) * pitch + st_id * 16, l0, l1, l2, l3,
+                    map_to_rank(bar(kBarMrg), static_cast<uint32_t>(i)));
+    }
+    // Then O^T, once every MMA has finished.  A split whose last commit never shows up sends NaN: the owner
+    // then recomputes the row on the exact path instead of dividing a short numerator by a full row sum.
+    bool have_o = have;
+    if (have_o) have_o = mbar_wait_warp(bar(kBarODone), 0, abort_flag);
     FALCON_TRACE(tid == 64, 44);
     tc_fence_after();
-    // Q, the ring and P^T are idle now (all of this CTA's MMAs have finished, all its loads landed).
-    if (n_splits > 1) cluster_wait();  // phase 1 (arrived long ago): every peer's merge barrier is initialised
-    // scratch for the row sums: inside ring stage 0, behind the staging rows
-    float* s_lpart = reinterpret_cast<float*>(smem_gen + off_kv + 16384);
+    // The ring and P^T are idle now (all of this CTA's MMAs have finished, all its loads landed).
     const uint32_t row_dst = slot_addr(o_me) + static_cast<uint32_t>(dl_me) * pitch;
     const uint32_t row_bar = map_to_rank(bar(kBarMrg), static_cast<uint32_t>(o_me));
 #pragma unroll
@@ -839,8 +868,8 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
       if (ch < n_chunks) {
         uint32_t o[kCW];
 #pragma unroll
-        for (int c = 0; c < kCW; ++c) o[c] = 0u;
-        if (have) {
+        for (int c = 0; c < kCW; ++c) o[c] = have ? 0x7fc00000u : 0u;
+        if (have_o) {
           tmem_ld_chunk<kCW>(tmem_lane + 2 * col_stride + ch * kCW, o);
           tmem_wait_ld();
         }
@@ -853,24 +882,7 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 #pragma unroll
         for (int u = 0; u < kCW / 8; ++u)
           st_async_v4(row_dst + ch * (kCW * 2) + u * 16, h[4 * u], h[4 * u + 1], h[4 * u + 2], h[4 * u + 3], row_bar);
-        // this warp's 32 keys' share of the chunk's row sums
-        const float sum = warp_col_sums<kCW>(l_acc[ci], lane);
-        if ((lane & (kCW == 16 ? 1 : 17)) == 0) s_lpart[q4 * C::kN + ch * kCW + col_of_lane<kCW>(lane)] = have ? sum : 0.f;
       }
-    }
-    // Row sums: the four lane quadrants' shares added (fixed order), four rows per thread, to every CTA
-    // (fp32, 4 bytes a query row, in the space of two more rows of the slot).
-    asm volatile("bar.sync 1, %0;" ::"n"(kSmThreads) : "memory");
-    if (st_id * 4 < N) {
-      const float4 s0 = reinterpret_cast<const float4*>(s_lpart)[st_id];
-      const float4 s1 = reinterpret_cast<const float4*>(s_lpart + C::kN)[st_id];
-      const float4 s2 = reinterpret_cast<const float4*>(s_lpart + 2 * C::kN)[st_id];
-      const float4 s3 = reinterpret_cast<const float4*>(s_lpart + 3 * C::kN)[st_id];
-      const uint32_t l0 = __float_as_uint((s0.x + s1.x) + (s2.x + s3.x)), l1 = __float_as_uint((s0.y + s1.y) + (s2.y + s3.y));
-      const uint32_t l2 = __float_as_uint((s0.z + s1.z) + (s2.z + s3.z)), l3 = __float_as_uint((s0.w + s1.w) + (s2.w + s3.w));
-      for (int i = 0; i < n_splits; ++i)
-        st_async_v4(slot_addr(i) + static_cast<uint32_t>(d_per) * pitch + st_id * 16, l0, l1, l2, l3,
-                    map_to_rank(bar(kBarMrg), static_cast<uint32_t>(i)));
     }
     FALCON_TRACE(tid == 64, 45);
   } 
@@ -913,7 +925,7 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     for (int c = 0; c < 4; ++c) {
       const int r = qc * 4 + c;
       if (r < n_valid) {
-        if (got && ls[c] >= kLMin && ls[c] <= kLMax) {
+        if (got && ls[c] >= kLMin && ls[c] <= kLMax && acc[c] == acc[c]) {
           const int mg = mtile * N + r;
           out_base[((mg >> p.g_shift) * p.Hq + (mg & (G - 1))) * kD + dl] = __float2bfloat16_rn(__fdividef(acc[c], ls[c]));
         } else if (dl == 0) {
