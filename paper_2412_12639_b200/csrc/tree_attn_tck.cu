@@ -363,6 +363,17 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
   const int G = p.G, N = p.n_rows, n_chunks = N / kCW;
   const uint32_t q_half_bytes = static_cast<uint32_t>(N) * 128u;  // between the two 64-column halves of Q
   FALCON_TRACE(tid == 0, 0);
+  if (warp == kWarpProducer) {
+    // the barriers first: their initialisation (and its fence) runs under the parameter reads below
+    if (lane == 0) {
+      *abort_flag = (smem_base & 1023u) ? 1 : 0;  // the swizzled tiles need a 1 KB aligned base
+      prefetch_tmap(&tm_k);
+      prefetch_tmap(&tm_v);
+    }
+    if (lane < kNumBars)
+      mbar_init(bar(lane), (lane == kBarPFull || lane == kBarPFull + 1 || lane == kBarQ) ? kSmWarps : 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
   {
     // The kernel's parameters live in constant memory that is rewritten for every launch, so the
     // first access to each of its 64-byte lines is a round trip to L2.  Touch every line now, where
@@ -456,14 +467,6 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     for (int i = st_id; i < 128 * static_cast<int>(C::kDescWords); i += kSmThreads) s_desc[i] = 0u;
     if (st_id < C::kN) s_rescue[st_id] = 0;
   } else if (warp == kWarpProducer) {
-    if (lane == 0) {
-      *abort_flag = (smem_base & 1023u) ? 1 : 0;  // the swizzled tiles need a 1 KB aligned base
-      prefetch_tmap(&tm_k);
-      prefetch_tmap(&tm_v);
-    }
-    if (lane < kNumBars)
-      mbar_init(bar(lane), (lane == kBarPFull || lane == kBarPFull + 1 || lane == kBarQ) ? kSmWarps : 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncwarp();
     FALCON_TRACE(tid == 0, 21);
     if (p.have_host && n_valid > 0 && lane == 0 && p.early_prefix) {
@@ -631,9 +634,8 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     FALCON_TRACE(tid == 64 && live && par_raw != 0x12345, 8);
     if (live) {
       // (a) Q block into shared memory in the layout the MMA reads (K-major rows of 128 bytes per
-      // 64-column half, 16-byte units XOR-swizzled by the row), and the reference of every query
-      // row: its scaled score against cache row 0 (8 threads per row, 16 columns each).
-      const uint32_t kw[8] = {kref[0].x, kref[0].y, kref[0].z, kref[0].w, kref[1].x, kref[1].y, kref[1].z, kref[1].w};
+      // 64-column half, 16-byte units XOR-swizzled by the row).  The MMA warp is told at once; the
+      // references below need cache row 0 as well, which arrives later, and nobody waits for them yet.
 #pragma unroll
       for (int pass = 0; pass < VT::kQPasses; ++pass) {
         const int r = (st_id >> 3) + VT::kRowsPerPass * pass;
@@ -642,6 +644,19 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
           const int u0 = 2 * (q_part & 3);
           *reinterpret_cast<uint4*>(qrow + ((u0 ^ (r & 7)) << 4)) = qreg[pass][0];
           *reinterpret_cast<uint4*>(qrow + (((u0 + 1) ^ (r & 7)) << 4)) = qreg[pass][1];
+        }
+      }
+      fence_async_smem();  // the MMA reads Q through the async proxy
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(kBarQ));
+      FALCON_TRACE(tid == 64, 9);
+      // the reference of every query row: its scaled score against cache row 0 (8 threads per row,
+      // 16 columns each)
+      const uint32_t kw[8] = {kref[0].x, kref[0].y, kref[0].z, kref[0].w, kref[1].x, kref[1].y, kref[1].z, kref[1].w};
+#pragma unroll
+      for (int pass = 0; pass < VT::kQPasses; ++pass) {
+        const int r = (st_id >> 3) + VT::kRowsPerPass * pass;
+        if (r < N) {
           const uint32_t qw[8] = {qreg[pass][0].x, qreg[pass][0].y, qreg[pass][0].z, qreg[pass][0].w,
                                   qreg[pass][1].x, qreg[pass][1].y, qreg[pass][1].z, qreg[pass][1].w};
           float d = 0.f;
@@ -656,10 +671,6 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
           if (q_part == 0) s_ref[r] = -d * p.scale_log2;
         }
       }
-      fence_async_smem();  // the MMA reads Q through the async proxy
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(kBarQ));
-      FALCON_TRACE(tid == 64, 9);
       // (b) the parent array, for the walks below
       if (need_tree && !p.tree_mask && st_id < T) {
         const bool okp = st_id == 0 ? par_raw == -1 : (par_raw >= 0 && par_raw < st_id);
