@@ -836,10 +836,12 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
       return map_to_rank(local, static_cast<uint32_t>(owner));
     };
     const bool have = live && n_my > 0 && !*abort_flag;
+    uint32_t own_l[4] = {0u, 0u, 0u, 0u};
     if (n_splits > 1) cluster_wait();  // phase 1 (arrived long ago): every peer's merge barrier is initialised
     // The row sums first: they are complete with the last tile's softmax pass and do not have to wait for the
-    // MMAs that are still running (Q is free by now: the last scores could only come after every QK product,
-    // so this split's own slot, which lies over Q, may be written).
+    // MMAs that are still running.  They go to the other CTAs at once; this CTA's own slot lies over Q and,
+    // where it is larger than Q, over the ring's first stage, which the last MMAs may still be reading: its
+    // copy of the sums is written with the rest of the slot, after them.
     float* s_lpart = reinterpret_cast<float*>(small + C::kOffLpart);
 #pragma unroll
     for (int ci = 0; ci < kPer; ++ci) {
@@ -861,8 +863,13 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
       const uint32_t l0 = __float_as_uint((s0.x + s1.x) + (s2.x + s3.x)), l1 = __float_as_uint((s0.y + s1.y) + (s2.y + s3.y));
       const uint32_t l2 = __float_as_uint((s0.z + s1.z) + (s2.z + s3.z)), l3 = __float_as_uint((s0.w + s1.w) + (s2.w + s3.w));
       for (int i = 0; i < n_splits; ++i)
-        st_async_v4(slot_addr(i) + static_cast<uint32_t>(d_per) * pitch + st_id * 16, l0, l1, l2, l3,
-                    map_to_rank(bar(kBarMrg), static_cast<uint32_t>(i)));
+        if (i != split)
+          st_async_v4(slot_addr(i) + static_cast<uint32_t>(d_per) * pitch + st_id * 16, l0, l1, l2, l3,
+                      map_to_rank(bar(kBarMrg), static_cast<uint32_t>(i)));
+      own_l[0] = l0;
+      own_l[1] = l1;
+      own_l[2] = l2;
+      own_l[3] = l3;
     }
     // Then O^T, once every MMA has finished.  A split whose last commit never shows up sends NaN: the owner
     // then recomputes the row on the exact path instead of dividing a short numerator by a full row sum.
@@ -871,6 +878,9 @@ tree_attn_tck_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     FALCON_TRACE(tid == 64, 44);
     tc_fence_after();
     // The ring and P^T are idle now (all of this CTA's MMAs have finished, all its loads landed).
+    if (st_id * 4 < N)
+      st_async_v4(slot_addr(split) + static_cast<uint32_t>(d_per) * pitch + st_id * 16, own_l[0], own_l[1], own_l[2], own_l[3],
+                  map_to_rank(bar(kBarMrg), static_cast<uint32_t>(split)));
     const uint32_t row_dst = slot_addr(o_me) + static_cast<uint32_t>(dl_me) * pitch;
     const uint32_t row_bar = map_to_rank(bar(kBarMrg), static_cast<uint32_t>(o_me));
 #pragma unroll
