@@ -74,6 +74,11 @@ int falcon_destroy(falcon_ctx* ctx);
 const char* falcon_status_string(int status);
 /* Text of the last CUDA error seen by this context ("" if none). */
 const char* falcon_last_error(const falcon_ctx* ctx);
+/* Test hook: fills the shared memory and the tensor memory of every SM with `pattern`
+ * (0xffffffff is a NaN as bf16 and as fp32), on `stream`.  A kernel launched afterwards that
+ * reads on-chip memory it has not written itself then shows it in its results, instead of
+ * working by the luck of what an earlier launch left there.  Harmless: plain stores. */
+int falcon_test_poison(falcon_ctx* ctx, uint32_t pattern, void* stream);
 /* Host check of one tree: FALCON_OK iff T in [1, FALCON_T_MAX], parent[0] == -1
  * and 0 <= parent[i] < i.  `parent` is a HOST pointer. */
 int falcon_tree_validate_host(const int32_t* parent, int32_t T);

@@ -106,6 +106,8 @@ def load_library():
         fn = getattr(lib, name)
         fn.argtypes = [C.c_void_p, C.POINTER(argt), C.c_void_p]
         fn.restype = C.c_int
+    lib.falcon_test_poison.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
+    lib.falcon_test_poison.restype = C.c_int
     lib.falcon_tree_attn_kernel.argtypes = [C.c_void_p, C.POINTER(AttnArgs)]
     lib.falcon_tree_attn_kernel.restype = C.c_int
     lib.falcon_tree_accept_static.argtypes = [C.POINTER(AcceptArgs), C.c_void_p]
@@ -219,6 +221,12 @@ class Context:
         rc = self._lib.falcon_lm_head_argmax(self._h, C.byref(args), _stream(stream))
         if check:
             self._check(rc, "falcon_lm_head_argmax")
+        return rc
+
+    def falcon_test_poison(self, pattern: int = 0xFFFFFFFF, stream=None) -> int:
+        """Test hook: every SM's shared and tensor memory filled with `pattern`."""
+        rc = self._lib.falcon_test_poison(self._h, pattern, _stream(stream))
+        self._check(rc, "falcon_test_poison")
         return rc
 
     def falcon_feature_gather(self, args: GatherArgs, stream=None, check: bool = True) -> int:

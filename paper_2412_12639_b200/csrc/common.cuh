@@ -49,6 +49,7 @@ int launch_kv_compact(falcon_ctx* ctx, const falcon_compact_args& a, cudaStream_
 int launch_feature_gather(falcon_ctx* ctx, const falcon_gather_args& a, cudaStream_t s);
 int check_gather_args(const falcon_gather_args& g, int max_tree);
 int launch_tree_topm(falcon_ctx* ctx, const falcon_topm_args& a, cudaStream_t s);
+int launch_test_poison(falcon_ctx* ctx, uint32_t pattern, cudaStream_t s);
 int launch_tree_search(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_t s);
 int launch_tree_sample(falcon_ctx* ctx, const falcon_accept_args& a, cudaStream_t s);
 int launch_lm_head_argmax(falcon_ctx* ctx, const falcon_lm_argmax_args& a, cudaStream_t s);

@@ -169,6 +169,11 @@ static int attn_plan(falcon_ctx* ctx, const falcon_attn_args* a, int* kernel) {
   }
 }
 
+int falcon_test_poison(falcon_ctx* ctx, uint32_t pattern, void* stream) {
+  if (!ctx) return FALCON_ERR_INVALID_ARG;
+  return launch_test_poison(ctx, pattern, static_cast<cudaStream_t>(stream));
+}
+
 int falcon_tree_attn_kernel(falcon_ctx* ctx, const falcon_attn_args* a) {
   int kernel = -1;
   return attn_plan(ctx, a, &kernel) == FALCON_OK ? kernel : -1;

@@ -756,6 +756,53 @@ def test_sample_rejects_bad_arguments():
     torch.cuda.synchronize()
 
 
+# ------------------------------------------------------------------------ on-chip memory left by earlier launches
+@pytest.mark.parametrize("pattern", [0xFFFFFFFF, 0x7F7F7F7F])
+def test_results_do_not_depend_on_what_shared_and_tensor_memory_held(pattern):
+    """Before every call the shared memory and the tensor memory of all SMs are filled with NaNs (all ones) or
+    with huge finite numbers: a kernel that reads a tile row, an accumulator column or a scratch word it has not
+    written itself computes with those instead of with what an earlier launch left, and shows it here."""
+    rng = np.random.default_rng(2718)
+    c = H.ctx()
+    cases = [(binding.ATTN_TCK, [16], [112], 1, 1, 1), (binding.ATTN_TCK, [60], [68], 2, 2, 1),
+             (binding.ATTN_TCK, [60], [300], 2, 2, 2), (binding.ATTN_TCK, [80], [700], 2, 2, 3),
+             (binding.ATTN_TCK, [64], [900], 8, 1, 4), (binding.ATTN_TCK, [7, 33], [0, 130], 2, 2, 0),
+             (binding.ATTN_TC, [60], [300], 2, 2, 2), (binding.ATTN_TC, [100], [40], 2, 1, 0),
+             (binding.ATTN_WARP, [15], [128], 4, 4, 0), (binding.ATTN_SIMT, [20], [77], 2, 2, 0)]
+    for kernel, sizes, prefs, Hq, Hkv, splits in cases:
+        tb, q, k, v = random_case(rng, sizes, prefs, Hq, Hkv, 128)
+        ref = oracle_attn(tb, Hq, Hkv, 128, q, k, v)
+        dt = H.DevTrees(tb)
+        c.falcon_test_poison(pattern)
+        out, rc = H.run_attn(dt, Hq, Hkv, 128, q, k, v, kernel=kernel, n_splits=splits)
+        assert rc == 0 and not dt.status.cpu().numpy().any()
+        H.assert_attn_close(out, ref, tb.node_off)
+    # the scan kernels and the LM head
+    x = rng.standard_normal((9, 5000)).astype(np.float32)
+    c.falcon_test_poison(pattern)
+    gv, gi, _ = H.run_topm(x, 20)
+    rv, ri = oracle.topm(x, 20)
+    np.testing.assert_array_equal(gi, ri)
+    np.testing.assert_array_equal(gv, rv)
+    fi = rng.integers(-3, 4, size=(70, 192))
+    wi = rng.integers(-3, 4, size=(1500, 192))
+    f, w = synth.f32_to_bf16_bits(fi.astype(np.float32)), synth.f32_to_bf16_bits(wi.astype(np.float32))
+    c.falcon_test_poison(pattern)
+    g, mx, status, rc = H.run_lm_argmax(f, w)
+    g_ref, best_ref = oracle.lm_head_argmax(f, w)
+    assert rc == 0 and status == 0
+    np.testing.assert_array_equal(g, g_ref)
+    np.testing.assert_array_equal(mx.astype(np.float64), best_ref)
+    tbt = H.make_trees([12, 30], [3, 9], rng, vocab=5000)
+    lg = rng.standard_normal((tbt.total_nodes, 5000)).astype(np.float32)
+    c.falcon_test_poison(pattern)
+    g, path, n_path, nxt = H.run_accept(H.DevTrees(tbt), lg)
+    np.testing.assert_array_equal(g, oracle.argmax(lg))
+    rp, rn, rt = oracle.tree_accept(tbt.node_off, tbt.parent, tbt.token, g)
+    np.testing.assert_array_equal(path, rp)
+    np.testing.assert_array_equal(n_path, rn)
+
+
 # ------------------------------------------------------------------------ LM-head argmax (Section 3.1, Eq. 6)
 def assert_lm_argmax(f, w, hidden=None, tol=None):
     """The kernel sums in fp32 in the tensor core's order, the oracle in double: the maximum itself must agree
