@@ -756,6 +756,39 @@ def test_sample_rejects_bad_arguments():
     torch.cuda.synchronize()
 
 
+# ------------------------------------------------------------------------ the first launch of a process
+FIRST_LAUNCH_SCRIPT = r"""
+import sys
+import numpy as np
+sys.path.insert(0, sys.argv[1]); sys.path.insert(0, sys.argv[1] + "/tests")
+import gpu_harness as H
+from test_gpu_parity import random_case, oracle_attn
+T, L, Hq, Hkv, splits, kernel = [int(x) for x in sys.argv[2:8]]
+rng = np.random.default_rng(T + L)
+tb, q, k, v = random_case(rng, [T], [L], Hq, Hkv, 128)
+ref = oracle_attn(tb, Hq, Hkv, 128, q, k, v)
+dt = H.DevTrees(tb)
+out, rc = H.run_attn(dt, Hq, Hkv, 128, q, k, v, kernel=kernel, n_splits=splits)   # the process's first launch
+assert rc == 0 and not dt.status.cpu().numpy().any()
+H.assert_attn_close(out, ref, tb.node_off)
+"""
+
+
+@pytest.mark.parametrize("T,L,Hq,Hkv,splits,kernel", [(16, 112, 1, 1, 1, binding.ATTN_TCK), (60, 1024, 2, 2, 4, binding.ATTN_TCK),
+                                                      (80, 300, 2, 2, 2, binding.ATTN_TCK), (128, 300, 2, 2, 3, binding.ATTN_TC)])
+def test_first_launch_of_a_process_is_right(T, L, Hq, Hkv, splits, kernel):
+    # every other test runs after earlier launches have warmed caches and left their data on the chip; here the
+    # call under test is the very first kernel of a fresh process (a case that once showed a write into a tile
+    # that the last MMAs were still reading, and only then)
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", FIRST_LAUNCH_SCRIPT, root] + [str(x) for x in (T, L, Hq, Hkv, splits, kernel)],
+                       capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
 # ------------------------------------------------------------------------ on-chip memory left by earlier launches
 @pytest.mark.parametrize("pattern", [0xFFFFFFFF, 0x7F7F7F7F])
 def test_results_do_not_depend_on_what_shared_and_tensor_memory_held(pattern):
