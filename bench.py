@@ -256,6 +256,46 @@ def time_topm(ctx, binding, torch, dev, stream, logits_h, peak, m=20, copies=20,
                          "traffic": None}}
 
 
+def time_sampled_accept(ctx, binding, torch, dev, stream, tree, tb, logits_h, peak, copies=20, reps=20):
+    """falcon_tree_accept with temperature 1 (non-greedy decoding: every node's token drawn from its softmax with a
+    caller-supplied uniform number) on the step's logits shape: `copies` distinct matrices (more than L2) in one
+    CUDA graph, replayed; CUDA events on the launching stream.  Not part of the step."""
+    N, V = logits_h.shape
+    B = tb.batch
+    src = torch.from_numpy(logits_h).to(dev)
+    mats = [src.clone() for _ in range(copies)]
+    g = torch.Generator(device=dev)
+    g.manual_seed(13)
+    u = torch.rand(N, device=dev, generator=g)
+    tok = torch.empty(N, dtype=torch.int32, device=dev)
+    path = torch.empty((B, 128), dtype=torch.int32, device=dev)
+    n_path = torch.empty(B, dtype=torch.int32, device=dev)
+    nxt = torch.empty(B, dtype=torch.int32, device=dev)
+    calls = [binding.accept_args(tree, V, x, V, tok, path, 128, n_path, nxt, temperature=1.0, uniforms=u) for x in mats]
+    with torch.cuda.stream(stream):
+        for a in calls:
+            ctx.falcon_tree_accept(a)       # the first call allocates scratch: before the capture
+        stream.synchronize()
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr, stream=stream):
+            for a in calls:
+                ctx.falcon_tree_accept(a)
+        for _ in range(3):
+            gr.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            gr.replay()
+        e1.record(stream)
+        stream.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (reps * copies)
+    nbytes = 4 * N * V + 4 * N
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"rows": N, "vocab": V, "temperature": 1.0, "us_per_call": us, "bytes_per_call": nbytes,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                         "traffic": None}}
+
+
 def time_lm_head(ctx, binding, torch, dev, stream, n_rows, hidden, vocab, peak, workload, reps=10):
     """falcon_lm_head_argmax (Section 3.1, Eq. 6: the LM head applied to the nodes' features, greedy token only)
     at the workload's shape, hidden = query heads x head_dim: two distinct random heads alternate (together more
@@ -484,6 +524,7 @@ def run_falcon(args):
 
     # ---------------- outside the step: the selection that grows the tree (the row next to the hot path) ----
     topm = time_topm(ctx, binding, torch, dev, stream, logits_h, peak) if world == 1 else None
+    sampled = time_sampled_accept(ctx, binding, torch, dev, stream, tree, tb, logits_h, peak) if world == 1 else None
     lm = (time_lm_head(ctx, binding, torch, dev, stream, tb.total_nodes, spec.n_q_heads * spec.head_dim, spec.vocab, peak,
                        args.workload) if world == 1 else None)
 
@@ -513,7 +554,7 @@ def run_falcon(args):
         "gpu_launches": args.steps * (NL + 2),
         "clocks": clocks,
         "cpu_baseline": cpu,
-        "extras": {"falcon_topm": topm, "falcon_lm_head_argmax": lm},
+        "extras": {"falcon_topm": topm, "falcon_lm_head_argmax": lm, "falcon_tree_accept_sampled": sampled},
         "wall_s_timed": t_wall,
     }
     print(json.dumps(line))
